@@ -1,0 +1,366 @@
+#!/usr/bin/env python
+"""Benchmark of the RBS-Attention prefill hot path on B200.
+
+One step = one pass of the whole path over one layer of the 128K Qwen3-30B-A3B attention shape
+(32 query / 4 KV heads, head_dim 128, block 128): rbs_block_stats -> rbs_select -> rbs_sparse_prefill.
+Prints ONE JSON line (rank 0).  `--impl reference` times the fp64 CPU oracle on a bounded sample instead.
+
+Usage: python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+With N > 1 (torchrun): every rank runs an independent replica (the path has no exchange step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+METRIC = "prefill_attention_ms_per_layer_128k"
+UNIT = "ms/layer"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], tflops=p["bf16_tflops"], tflops_sustained=p.get("bf16_tflops_sustained"),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, tflops=1590.0, tflops_sustained=1400.0, source="fallback")
+
+
+def workload(name: str):
+    from paper_2609_20971_b200.synth import paper_configs
+    return paper_configs()[name]
+
+
+# ------------------------------------------------------------------------------------------------
+# clocks sampled during the timed region
+# ------------------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        self.lines = []
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100", "-i", str(index)],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.2] or [l for (_, l) in self.lines]
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for l in rows:
+            parts = [x.strip() for x in l.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------------------------
+# CPU oracle leg (cpu_baseline and --impl reference)
+# ------------------------------------------------------------------------------------------------
+def oracle_sample_ms_per_layer(cfg, Q, K, V, n_heads=1, n_att_rows=24):
+    """Times the oracle as it stands on a bounded sample of one layer and extrapolates to ms/layer.
+    Sample: block statistics of KV head 0 (all blocks), selection of `n_heads` query heads (all query
+    blocks), attention of `n_att_rows` query blocks of head 0; each part is scaled by the ratio of its
+    work units (blocks, heads, selected block pairs) to the layer's."""
+    from oracle import rbs_oracle as orc
+    from paper_2609_20971_b200.synth import to_f64
+    G = cfg.Hq // cfg.Hkv
+    M, B = cfg.M, cfg.B
+    K0 = to_f64(K[0, :, 0])
+    t = time.perf_counter()
+    c, r = orc.block_stats(K0, B)
+    beta, _, _ = orc.rescue_coefficient(r)
+    t_stats = (time.perf_counter() - t) * cfg.Hkv
+    t = time.perf_counter()
+    sels = []
+    for h in range(n_heads):
+        sels.append(orc.select_head(to_f64(Q[0, :, h]), c, r, beta, B, cfg.alpha_base, cfg.alpha_rescue,
+                                    cfg.n_sink, cfg.n_local, cfg.n_recent))
+    t_select = (time.perf_counter() - t) * cfg.Hq / n_heads
+    sel = sels[0]
+    rows = sorted({int(x) for x in np.linspace(0, M - 1, n_att_rows)})
+    Q0, V0 = to_f64(Q[0, :, 0]), to_f64(V[0, :, 0])
+    t = time.perf_counter()
+    pairs = 0
+    for i in rows:
+        orc.masked_attention_block(Q0, K0, V0, sel.final[i], i, B)
+        pairs += int(sel.final[i].sum())
+    dt = time.perf_counter() - t
+    total_pairs = sel.density * M * (M + 1) / 2 * cfg.Hq
+    t_att = dt * total_pairs / max(pairs, 1)
+    ms = (t_stats + t_select + t_att) * 1e3
+    sample = (f"stats: KV head 0 of {cfg.Hkv}; select: {n_heads} of {cfg.Hq} query heads, all {M} query blocks; "
+              f"attention: {len(rows)} query blocks of head 0 ({pairs} of ~{int(total_pairs)} selected pairs); "
+              "each part scaled linearly to one layer (extrapolated)")
+    return ms, sample, dict(stats_ms=t_stats * 1e3, select_ms=t_select * 1e3, attention_ms=t_att * 1e3,
+                            density_head0=sel.density)
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2609_20971_b200.synth import make_inputs
+    cfg = workload(args.workload)
+    Q, K, V = make_inputs(cfg)
+    cores = torch.get_num_threads()
+    for _ in range(args.warmup):
+        oracle_sample_ms_per_layer(cfg, Q, K, V, n_heads=1, n_att_rows=4)
+    vals, sample = [], ""
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        ms, sample, _ = oracle_sample_ms_per_layer(cfg, Q, K, V, n_heads=1, n_att_rows=8)
+        vals.append(ms)
+    wall = (time.perf_counter() - t0) * 1e3 / max(args.steps, 1)
+    value = float(np.mean(vals))
+    out = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": wall, "higher_is_better": False,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": cfg.name, **cfg.describe()},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out))
+
+
+# ------------------------------------------------------------------------------------------------
+# CUDA leg
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch.distributed as dist
+    from paper_2609_20971_b200 import alloc_stats, rbs_block_stats, rbs_select, rbs_sparse_prefill, workspace_bytes
+    from paper_2609_20971_b200.binding import RBS_OP_SELECT, RbsShape
+    from paper_2609_20971_b200.synth import make_inputs
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU fallback (use --impl reference for the oracle)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = load_peaks()
+    cfg = workload(args.workload)
+    cfg.seed += rank                       # independent replica per rank
+    Q, K, V = make_inputs(cfg)
+    Qh, Kh, Vh = Q.pin_memory(), K.pin_memory(), V.pin_memory()
+    Oh = torch.empty_like(Qh).pin_memory()
+    Qg, Kg, Vg = Qh.to(dev), Kh.to(dev), Vh.to(dev)
+    Og = torch.empty_like(Qg)
+    M, B, L = cfg.M, cfg.B, cfg.L
+    W = (M + 31) // 32
+    stats = alloc_stats(Kg, B)
+    mask = torch.empty(L, cfg.Hq, M, W, dtype=torch.int32, device=dev)
+    density = torch.empty(L, cfg.Hq, dtype=torch.float32, device=dev)
+    shape = RbsShape(L, cfg.N, cfg.Hq, cfg.Hkv, cfg.d, B)
+    ws = torch.empty(workspace_bytes(RBS_OP_SELECT, shape), dtype=torch.uint8, device=dev)
+    sel_args = (cfg.alpha_base, cfg.alpha_rescue, cfg.n_sink, cfg.n_local, cfg.n_recent)
+    stream = torch.cuda.current_stream()
+
+    def step(events=None):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)] if events is not None else None
+        if ev: ev[0].record(stream)
+        rbs_block_stats(Kg, B, stats)
+        if ev: ev[1].record(stream)
+        rbs_select(Qg, stats, B, *sel_args, mask=mask, density=density, workspace=ws)
+        if ev: ev[2].record(stream)
+        rbs_sparse_prefill(Qg, Kg, Vg, mask, B, out=Og)
+        if ev:
+            ev[3].record(stream)
+            events.append(ev)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    events = []
+    t_wall0 = time.time()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(args.steps):
+        step(events)
+    e1.record(stream)
+    barrier()
+    t_wall1 = time.time()
+    total_ms = e0.elapsed_time(e1)
+    clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    t_stats = statistics.mean(ev[0].elapsed_time(ev[1]) for ev in events)
+    t_select = statistics.mean(ev[1].elapsed_time(ev[2]) for ev in events)
+    t_sparse = statistics.mean(ev[2].elapsed_time(ev[3]) for ev in events)
+
+    # end to end: pinned host buffers -> device, the three calls, result back to the host
+    def e2e_step():
+        Qg.copy_(Qh, non_blocking=True); Kg.copy_(Kh, non_blocking=True); Vg.copy_(Vh, non_blocking=True)
+        step()
+        Oh.copy_(Og, non_blocking=True)
+    e2e_step()
+    barrier()
+    n_e2e = max(2, min(args.steps, 5))
+    e0.record(stream)
+    for _ in range(n_e2e):
+        e2e_step()
+    e1.record(stream)
+    barrier()
+    e2e_ms = e0.elapsed_time(e1) / n_e2e
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    h2d = Qh.numel() * 2 + Kh.numel() * 2 + Vh.numel() * 2
+    d2h = Oh.numel() * 2
+
+    # dense baseline on the same inputs (the same kernel with every causal block selected)
+    n_dense = 2
+    rbs_sparse_prefill(Qg, Kg, Vg, None, B, out=Og)
+    barrier()
+    e0.record(stream)
+    for _ in range(n_dense):
+        rbs_sparse_prefill(Qg, Kg, Vg, None, B, out=Og)
+    e1.record(stream)
+    barrier()
+    t_dense = e0.elapsed_time(e1) / n_dense
+
+    # stats pass alone over rotating K copies (K of one layer is about the size of L2)
+    n_rot = 4
+    Krot = [Kg] + [Kg.clone() for _ in range(n_rot - 1)]
+    for k in Krot:
+        rbs_block_stats(k, B, stats)
+    barrier()
+    reps = 5
+    e0.record(stream)
+    for _ in range(reps):
+        for k in Krot:
+            rbs_block_stats(k, B, stats)
+    e1.record(stream)
+    barrier()
+    t_stats_rot = e0.elapsed_time(e1) / (reps * n_rot)
+    del Krot
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    dens = density.float().cpu().numpy().astype(np.float64)
+    pairs_all = M * (M + 1) // 2
+    sel_pairs = float((dens * pairs_all).sum())                  # over L x Hq
+    diag_pairs = float(L * cfg.Hq * M)                           # the diagonal is always kept (n_local >= 1)
+    flop_pair = 4.0 * B * B * cfg.d
+    useful = flop_pair * ((sel_pairs - diag_pairs) + diag_pairs * (B + 1) / (2.0 * B))
+    executed = flop_pair * sel_pairs
+    dense_useful = flop_pair * L * cfg.Hq * ((pairs_all - M) + M * (B + 1) / (2.0 * B))
+    tflops_sparse = useful / (t_sparse * 1e-3) / 1e12
+    stats_bytes = Kg.numel() * 2 + stats.centroid.numel() * 4 + stats.radius.numel() * 4
+    stats_gbs = stats_bytes / (t_stats_rot * 1e-3) / 1e9
+
+    cpu_ms, cpu_sample, cpu_parts = (None, None, None)
+    if world == 1 and not args.no_cpu_baseline:
+        cfg0 = workload(args.workload)
+        cpu_ms, cpu_sample, cpu_parts = oracle_sample_ms_per_layer(cfg0, Q, K, V, n_heads=1, n_att_rows=24)
+
+    value = ms_per_step / (world * L)
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": cfg.name, "l2": "inputs larger than L2 (Q+O 2 GiB per step)", **cfg.describe()},
+        "roofline": {"bound": "tensor", "kernel": "rbs_sparse_prefill", "achieved": tflops_sparse,
+                     "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": tflops_sparse / peaks["tflops"],
+                     "traffic": None, "peak_source": peaks["source"],
+                     "flops_per_launch_useful": useful, "flops_per_launch_executed": executed},
+        "cpu_baseline": ({"value": cpu_ms, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
+                          "sample": cpu_sample, "parts": cpu_parts} if cpu_ms is not None else None),
+        "e2e": {"value": e2e_ms / (world * L), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "gpu_launches": 6 * args.steps,
+        "clocks": clocks,
+        "detail": {
+            "t_stats_ms": t_stats, "t_select_ms": t_select, "t_sparse_ms": t_sparse, "t_dense_ms": t_dense,
+            "speedup_vs_dense": t_dense / (t_select + t_sparse),
+            "speedup_vs_dense_incl_stats": t_dense / (t_stats + t_select + t_sparse),
+            "density_mean": float(dens.mean()), "density_min": float(dens.min()), "density_max": float(dens.max()),
+            "selected_tflop_useful": useful / 1e12,
+            "tensor_frac_select_plus_sparse": useful / ((t_select + t_sparse) * 1e-3) / 1e12 / peaks["tflops"],
+            "dense_tflops": dense_useful / (t_dense * 1e-3) / 1e12,
+            "dense_tensor_frac": dense_useful / (t_dense * 1e-3) / 1e12 / peaks["tflops"],
+            "stats_rotating_us": t_stats_rot * 1e3, "stats_gbs": stats_gbs, "stats_hbm_frac": stats_gbs / peaks["hbm_gbs"],
+            "peaks": peaks,
+        },
+    }
+    print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="q30b_128k")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

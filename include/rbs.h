@@ -1,0 +1,138 @@
+/*
+ * rbs.h -- C ABI of the RBS-Attention prefill hot path for NVIDIA B200 (sm_100a).
+ *
+ * Three calls per layer follow Algorithm 1 of the paper:
+ *   rbs_block_stats     key-block centroids and radii                    (Sec. 3.1)
+ *   rbs_select          rescue coefficients, dual-branch block selection (Sec. 3.1-3.2)
+ *   rbs_sparse_prefill  causal block-sparse attention over the mask      (Sec. 3.3, Eq. 1 when dense)
+ *
+ * Conventions for every entry point
+ *   - All data pointers are DEVICE pointers unless a parameter says "host".  The caller owns every
+ *     buffer; the library allocates nothing on these paths and keeps no state between calls.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the legacy default
+ *     stream) and the call returns without waiting for it.
+ *   - Argument errors are detected on the host before anything is launched and reported through
+ *     the return value; nothing is written in that case.  There is no CPU fallback.
+ *   - Q/K/V/O are bf16 tensors with the head dimension contiguous, addressed as
+ *       element(l, t, h, j) = ptr[l*stride_batch + t*stride_token + h*stride_head + j]
+ *     (strides in elements, multiples of 8; ptr 16-byte aligned).  The natural layout is
+ *     [batch][token][head][head_dim].  `batch` is prompts x layers: every (batch, KV head) is an
+ *     independent problem.
+ *   - Notation: N = seqlen, B = block, M = N / B blocks, Hq / Hkv query / KV heads,
+ *     G = Hq / Hkv, query head h reads KV head h / G, d = head_dim, W = ceil(M / 32).
+ *   - Supported: head_dim == 128, block in {64, 128}, seqlen a positive multiple of block,
+ *     Hq a multiple of Hkv, M <= 8192.  Anything else returns RBS_ERR_UNSUPPORTED.
+ */
+#ifndef RBS_H_
+#define RBS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define RBS_API __attribute__((visibility("default")))
+#else
+#define RBS_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  RBS_OK = 0,
+  RBS_ERR_INVALID_ARG = 1, /* null pointer, misaligned pointer or stride, alpha <= 0, negative count */
+  RBS_ERR_UNSUPPORTED = 2, /* shape outside the supported set listed above */
+  RBS_ERR_WORKSPACE = 3,   /* workspace missing or smaller than rbs_workspace_bytes() */
+  RBS_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (launch, tensor-map encode, ...) */
+  RBS_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up  */
+} rbs_status;
+
+typedef struct {
+  int batch;      /* L: prompts x layers */
+  int seqlen;     /* N */
+  int n_q_heads;  /* Hq */
+  int n_kv_heads; /* Hkv */
+  int head_dim;   /* d */
+  int block;      /* B: block size of queries and of keys (Sec. 4.4: 128 by default) */
+} rbs_shape;
+
+typedef struct {
+  void* ptr;            /* device, bf16 */
+  int64_t stride_batch; /* elements */
+  int64_t stride_token;
+  int64_t stride_head;
+} rbs_tensor;
+
+/* Per-block key statistics (Sec. 3.1), all device fp32, dense row-major in the index order shown. */
+typedef struct {
+  float* centroid; /* [L][Hkv][M][d]  c_b = mean of the block's keys */
+  float* radius;   /* [L][Hkv][M]     r_b = max_k ||k - c_b||_2 */
+  float* beta;     /* [L][Hkv][M]     rescue coefficient, Eq. (beta) */
+  float* rq;       /* [L][Hkv][2]     (r_low, r_high) = radius quantiles 0.5 and 0.9 */
+} rbs_stats;
+
+enum { RBS_OP_BLOCK_STATS = 0, RBS_OP_SELECT = 1, RBS_OP_SPARSE_PREFILL = 2 };
+
+/* Bytes of device workspace the given call needs for this shape (0 if none).  Workspace must be
+ * 256-byte aligned; its contents need not be initialised and are undefined afterwards. */
+RBS_API size_t rbs_workspace_bytes(int op, const rbs_shape* shape);
+
+/*
+ * Sec. 3.1 / Algorithm 1, first loop.  Reads K once and writes, for every (l, KV head, block b),
+ *   stats.centroid = (1/B) sum of the block's keys                  (fp32 accumulation of bf16 keys)
+ *   stats.radius   = max over the block's keys of ||k - c_b||_2     (difference form, fp32)
+ * stats.beta and stats.rq are not touched.  Needs no workspace.
+ */
+RBS_API rbs_status rbs_block_stats(const rbs_shape* shape, rbs_tensor K, rbs_stats stats, void* stream);
+
+/*
+ * Sec. 3.1-3.2 / Algorithm 1, second and third loops.
+ *   1. per (l, KV head): r_low = quantile(r, 0.5), r_high = quantile(r, 0.9) (linear interpolation
+ *      between order statistics at p*(M-1)); beta_b = clamp((r_b - r_low)/(r_high - r_low), 0, 1),
+ *      beta = 0 when r_high <= r_low.  Written to stats.rq and stats.beta.
+ *   2. per (l, query head h, query block i), for every causal key block b <= i:
+ *        S_base[i,b]   = sum_{t in Q_i} exp( q_t.c_b / sqrt(d) - m )
+ *        S_rescue[i,b] = sum_{t in Q_i} exp((q_t.c_b + ||q_t|| r_b beta_b) / sqrt(d) - m')
+ *      (Eq. base_score, rescue_score, block_aggregation; evaluated as per-block log-sum-exp), then
+ *        keep b  iff  S_base >= alpha_base * max_b' S_base   or   S_rescue >= alpha_rescue * max_b' S_rescue
+ *        or b is forced: b < n_sink, or i - n_local < b <= i, or i >= M - n_recent
+ *      (Eq. branch_thresholds and the mask union).
+ *   3. density[l][h] = kept causal pairs / (M (M+1) / 2)              (Eq. actual_density).
+ * stats.centroid and stats.radius are inputs (from rbs_block_stats).
+ * mask: uint32 [L][Hq][M][W]; key block b of query block i is bit (b % 32) of word b / 32; bits
+ *   with b > i are written as 0.  dbg_base_mask / dbg_rescue_mask (same layout) receive the two
+ *   branch masks before the union when non-NULL.
+ * alpha > 1 disables that branch (empty set).  alpha must be > 0.
+ * Workspace: rbs_workspace_bytes(RBS_OP_SELECT, shape).
+ */
+RBS_API rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats stats, float alpha_base,
+                      float alpha_rescue, int n_sink, int n_local, int n_recent, uint32_t* mask,
+                      float* density, uint32_t* dbg_base_mask, uint32_t* dbg_rescue_mask,
+                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Sec. 3.3 / Algorithm 1, last step; Eq. (1) when mask == NULL.
+ * For token t of query block i and query head h:
+ *   O_t = sum_j softmax_j(q_t.k_j * scale) v_j  over keys j <= t whose block is set in mask row (l,h,i),
+ * the softmax normalised over those retained keys only.  bf16 inputs, fp32 accumulation and
+ * softmax, bf16 output.  mask == NULL selects every causal block (the dense baseline, density 1).
+ * Mask bits with b > i are ignored.  A row with no retained key outputs zeros and lse = -inf.
+ * lse (nullable): fp32 [L][Hq][N], natural-log-sum-exp of the scaled retained logits.
+ * softmax_scale == 0 means 1/sqrt(d).
+ * Workspace: rbs_workspace_bytes(RBS_OP_SPARSE_PREFILL, shape).
+ */
+RBS_API rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, rbs_tensor K, rbs_tensor V,
+                              const uint32_t* mask, rbs_tensor O, float* lse, float softmax_scale,
+                              void* workspace, size_t workspace_bytes, void* stream);
+
+/* Human-readable name of a status code (static storage, never NULL). */
+RBS_API const char* rbs_status_string(rbs_status status);
+
+/* Library version string (static storage), e.g. for logging next to measurements. */
+RBS_API const char* rbs_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RBS_H_ */

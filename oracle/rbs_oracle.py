@@ -156,10 +156,12 @@ class HeadSelection:
 
 def select_head(Q: np.ndarray, centroid: np.ndarray, radius: np.ndarray, beta: np.ndarray,
                 block: int, alpha_base: float, alpha_rescue: float,
-                n_sink: int, n_local: int, n_recent: int) -> HeadSelection:
+                n_sink: int, n_local: int, n_recent: int, rows=None) -> HeadSelection:
     """Algorithm 1, third loop, for ONE query head against its KV head's statistics.
 
     Q [N, d]; centroid [M, d]; radius, beta [M].  N must be a multiple of `block`.
+    `rows` (optional) restricts the work to those query blocks; other rows stay empty and the
+    returned density is then meaningless.
     """
     Q = np.asarray(Q, dtype=np.float64)
     N, d = Q.shape
@@ -170,7 +172,7 @@ def select_head(Q: np.ndarray, centroid: np.ndarray, radius: np.ndarray, beta: n
     forced = np.zeros((M, M), dtype=bool)
     margin_base = np.full((M, M), np.inf)
     margin_rescue = np.full((M, M), np.inf)
-    for i in range(M):
+    for i in (range(M) if rows is None else rows):
         Qi = Q[i * block:(i + 1) * block]
         nb = i + 1  # causal candidates C_i = {0..i}
         l_base, l_rescue = branch_logits(Qi, centroid[:nb], radius[:nb], beta[:nb])

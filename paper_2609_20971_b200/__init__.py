@@ -1,0 +1,11 @@
+"""RBS-Attention prefill hot path for NVIDIA B200: block statistics, dual-branch block selection and
+causal block-sparse attention as hand-written sm_100a kernels behind a small C ABI (include/rbs.h).
+
+The Python names mirror the C entry points.  Importing this package does not load the CUDA library;
+the first call does, and raises if it has not been built.
+"""
+from .binding import (BlockStats, RbsError, alloc_stats, load_library, rbs_block_stats, rbs_select,
+                      rbs_sparse_prefill, workspace_bytes)
+
+__all__ = ["BlockStats", "RbsError", "alloc_stats", "load_library", "rbs_block_stats", "rbs_select",
+           "rbs_sparse_prefill", "workspace_bytes"]

@@ -1,0 +1,175 @@
+"""Thin ctypes binding over the C ABI declared in include/rbs.h.
+
+Argument marshalling only: tensor pointers, strides and the current CUDA stream are handed to the
+library; every step of the path runs in the library's kernels.  torch provides device memory and
+streams.  There is no fallback: if the shared library is missing or a call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "librbs_b200.so")
+
+RBS_OP_BLOCK_STATS, RBS_OP_SELECT, RBS_OP_SPARSE_PREFILL = 0, 1, 2
+
+
+class RbsShape(ctypes.Structure):
+    _fields_ = [("batch", ctypes.c_int), ("seqlen", ctypes.c_int), ("n_q_heads", ctypes.c_int),
+                ("n_kv_heads", ctypes.c_int), ("head_dim", ctypes.c_int), ("block", ctypes.c_int)]
+
+
+class RbsTensor(ctypes.Structure):
+    _fields_ = [("ptr", ctypes.c_void_p), ("stride_batch", ctypes.c_int64),
+                ("stride_token", ctypes.c_int64), ("stride_head", ctypes.c_int64)]
+
+
+class RbsStats(ctypes.Structure):
+    _fields_ = [("centroid", ctypes.c_void_p), ("radius", ctypes.c_void_p),
+                ("beta", ctypes.c_void_p), ("rq", ctypes.c_void_p)]
+
+
+class RbsError(RuntimeError):
+    pass
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the CUDA library built by build.py; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RbsError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_20971_b200.build` "
+                       "(there is no CPU fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, sz, f, i = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_float, ctypes.c_int
+    lib.rbs_workspace_bytes.restype = sz
+    lib.rbs_workspace_bytes.argtypes = [i, ctypes.POINTER(RbsShape)]
+    lib.rbs_block_stats.restype = i
+    lib.rbs_block_stats.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, vp]
+    lib.rbs_select.restype = i
+    lib.rbs_select.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, f, f, i, i, i, vp, vp, vp, vp, vp, sz, vp]
+    lib.rbs_sparse_prefill.restype = i
+    lib.rbs_sparse_prefill.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsTensor, RbsTensor, vp, RbsTensor,
+                                       vp, f, vp, sz, vp]
+    lib.rbs_status_string.restype = ctypes.c_char_p
+    lib.rbs_status_string.argtypes = [i]
+    lib.rbs_version.restype = ctypes.c_char_p
+    lib.rbs_version.argtypes = []
+    _lib = lib
+    return lib
+
+
+def _check(code: int, what: str) -> None:
+    if code != 0:
+        raise RbsError(f"{what} failed: {load_library().rbs_status_string(code).decode()}")
+
+
+def _tensor(t: torch.Tensor) -> RbsTensor:
+    if t.dim() != 4 or t.dtype != torch.bfloat16 or not t.is_cuda or t.stride(3) != 1:
+        raise RbsError("expected a CUDA bf16 tensor [batch, tokens, heads, head_dim] with head_dim contiguous")
+    return RbsTensor(t.data_ptr(), t.stride(0), t.stride(1), t.stride(2))
+
+
+def _shape(Q_or_none, K, block: int, n_q_heads: int | None = None) -> RbsShape:
+    L, N, Hkv, d = K.shape
+    Hq = n_q_heads if n_q_heads is not None else (Q_or_none.shape[2] if Q_or_none is not None else Hkv)
+    return RbsShape(L, N, Hq, Hkv, d, block)
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _ptr(t) -> ctypes.c_void_p:
+    return ctypes.c_void_p(None if t is None else t.data_ptr())
+
+
+@dataclass
+class BlockStats:
+    centroid: torch.Tensor  # [L, Hkv, M, d] fp32
+    radius: torch.Tensor    # [L, Hkv, M]    fp32
+    beta: torch.Tensor      # [L, Hkv, M]    fp32, written by rbs_select
+    rq: torch.Tensor        # [L, Hkv, 2]    fp32, written by rbs_select
+
+    def c_struct(self) -> RbsStats:
+        return RbsStats(self.centroid.data_ptr(), self.radius.data_ptr(), self.beta.data_ptr(), self.rq.data_ptr())
+
+
+def alloc_stats(K: torch.Tensor, block: int) -> BlockStats:
+    L, N, Hkv, d = K.shape
+    M = N // block
+    dev = K.device
+    return BlockStats(torch.empty(L, Hkv, M, d, dtype=torch.float32, device=dev),
+                      torch.empty(L, Hkv, M, dtype=torch.float32, device=dev),
+                      torch.zeros(L, Hkv, M, dtype=torch.float32, device=dev),
+                      torch.zeros(L, Hkv, 2, dtype=torch.float32, device=dev))
+
+
+def workspace_bytes(op: int, shape: RbsShape) -> int:
+    return int(load_library().rbs_workspace_bytes(op, ctypes.byref(shape)))
+
+
+def rbs_block_stats(K: torch.Tensor, block: int, stats: BlockStats | None = None) -> BlockStats:
+    """Key-block centroids and radii (Sec. 3.1).  K: [L, N, Hkv, d] bf16 on the GPU."""
+    lib = load_library()
+    if stats is None:
+        stats = alloc_stats(K, block)
+    shape = _shape(None, K, block)
+    _check(lib.rbs_block_stats(ctypes.byref(shape), _tensor(K), stats.c_struct(), _stream()), "rbs_block_stats")
+    return stats
+
+
+def rbs_select(Q: torch.Tensor, stats: BlockStats, block: int, alpha_base: float = 0.22, alpha_rescue: float = 0.18,
+               n_sink: int = 1, n_local: int = 1, n_recent: int = 1, *, mask: torch.Tensor | None = None,
+               density: torch.Tensor | None = None, workspace: torch.Tensor | None = None, debug: bool = False):
+    """Dual-branch block selection (Sec. 3.2).  Returns (mask uint32-as-int32 [L,Hq,M,W], density [L,Hq])
+    and, with debug=True, also the base and rescue branch masks."""
+    lib = load_library()
+    L, N, Hq, d = Q.shape
+    Hkv = stats.centroid.shape[1]
+    M = N // block
+    W = (M + 31) // 32
+    shape = RbsShape(L, N, Hq, Hkv, d, block)
+    dev = Q.device
+    if mask is None:
+        mask = torch.empty(L, Hq, M, W, dtype=torch.int32, device=dev)
+    if density is None:
+        density = torch.empty(L, Hq, dtype=torch.float32, device=dev)
+    need = workspace_bytes(RBS_OP_SELECT, shape)
+    if workspace is None:
+        workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
+    dbg_b = torch.empty_like(mask) if debug else None
+    dbg_r = torch.empty_like(mask) if debug else None
+    _check(lib.rbs_select(ctypes.byref(shape), _tensor(Q), stats.c_struct(), alpha_base, alpha_rescue,
+                          n_sink, n_local, n_recent, _ptr(mask), _ptr(density), _ptr(dbg_b), _ptr(dbg_r),
+                          _ptr(workspace), workspace.numel(), _stream()), "rbs_select")
+    if debug:
+        return mask, density, dbg_b, dbg_r
+    return mask, density
+
+
+def rbs_sparse_prefill(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, mask: torch.Tensor | None, block: int, *,
+                       out: torch.Tensor | None = None, return_lse: bool = False, softmax_scale: float = 0.0,
+                       workspace: torch.Tensor | None = None):
+    """Causal block-sparse attention over `mask` (Sec. 3.3); mask=None is dense causal attention (Eq. 1)."""
+    lib = load_library()
+    L, N, Hq, d = Q.shape
+    shape = RbsShape(L, N, Hq, K.shape[2], d, block)
+    if out is None:
+        out = torch.empty_like(Q)
+    lse = torch.empty(L, Hq, N, dtype=torch.float32, device=Q.device) if return_lse else None
+    need = workspace_bytes(RBS_OP_SPARSE_PREFILL, shape)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=Q.device)
+    _check(lib.rbs_sparse_prefill(ctypes.byref(shape), _tensor(Q), _tensor(K), _tensor(V), _ptr(mask), _tensor(out),
+                                  _ptr(lse), softmax_scale, _ptr(workspace),
+                                  0 if workspace is None else workspace.numel(), _stream()), "rbs_sparse_prefill")
+    return (out, lse) if return_lse else out

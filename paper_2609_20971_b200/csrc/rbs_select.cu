@@ -1,0 +1,351 @@
+// rbs_select: rescue coefficients (Eq. beta), dual-branch block scores (Eq. base_score, rescue_score,
+// block_aggregation), per-branch relative thresholds, forced blocks, union, bit-packed mask, density.
+//
+// Scoring works on the transposed product  X^T = C . Q_i^T  (centroids are the M-dimension, the tokens of
+// the query block the N-dimension) so that the sum over tokens needed by the aggregation runs along the
+// accumulator row of one centroid.  Centroids are fed to the tensor cores as bf16 hi + bf16 lo
+// (two accumulating products) so that the logit keeps ~16 mantissa bits of the fp32 centroid.
+// Scores are kept per block as log2-sum-exp2, L = log2 sum_t 2^(z_t); the relative threshold
+// S >= alpha max S becomes L >= log2(alpha) + max L (the common shift of Eq. block_aggregation cancels).
+#include "rbs_common.cuh"
+
+namespace rbs {
+
+// ---------------------------------------------------------------------------------------------
+// 1. per (l, KV head): sort radii, quantiles, beta, g = r * beta * scale * log2(e)
+// ---------------------------------------------------------------------------------------------
+constexpr int kCoeffThreads = 1024;
+
+__global__ void __launch_bounds__(kCoeffThreads)
+rescue_coeff_kernel(const float* __restrict__ radius, int M, int P /* pow2 >= M */, float scale_log2,
+                    float* __restrict__ beta, float* __restrict__ rq, float* __restrict__ g, int Mpad) {
+  extern __shared__ float s_sorted[];
+  __shared__ float s_q[2];
+  const int hd = blockIdx.x, tid = threadIdx.x;
+  const float* r = radius + static_cast<int64_t>(hd) * M;
+  for (int idx = tid; idx < P; idx += kCoeffThreads) s_sorted[idx] = idx < M ? r[idx] : __int_as_float(0x7f800000);
+  __syncthreads();
+  for (int k = 2; k <= P; k <<= 1) {
+    for (int j = k >> 1; j > 0; j >>= 1) {
+      for (int idx = tid; idx < P; idx += kCoeffThreads) {
+        const int ixj = idx ^ j;
+        if (ixj > idx) {
+          const float a = s_sorted[idx], c = s_sorted[ixj];
+          const bool asc = (idx & k) == 0;
+          if ((a > c) == asc) { s_sorted[idx] = c; s_sorted[ixj] = a; }
+        }
+      }
+      __syncthreads();
+    }
+  }
+  if (tid < 2) {
+    // quantile(p): linear interpolation between order statistics at position p (M - 1)
+    const double p = tid == 0 ? 0.5 : 0.9;
+    const double x = p * static_cast<double>(M - 1);
+    const int lo = static_cast<int>(floor(x));
+    const int hi = min(lo + 1, M - 1);
+    const double a = static_cast<double>(s_sorted[lo]), c = static_cast<double>(s_sorted[hi]);
+    const float q = static_cast<float>(a + (x - lo) * (c - a));
+    s_q[tid] = q;
+    rq[hd * 2 + tid] = q;
+  }
+  __syncthreads();
+  const float r_low = s_q[0], r_high = s_q[1];
+  const bool live = r_high > r_low;
+  const float inv = live ? 1.0f / (r_high - r_low) : 0.f;
+  for (int idx = tid; idx < Mpad; idx += kCoeffThreads) {
+    float bt = 0.f, rb = 0.f;
+    if (idx < M) {
+      rb = r[idx];
+      bt = live ? fminf(fmaxf((rb - r_low) * inv, 0.f), 1.f) : 0.f;
+      beta[static_cast<int64_t>(hd) * M + idx] = bt;
+    }
+    g[static_cast<int64_t>(hd) * Mpad + idx] = rb * bt * scale_log2;
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// 2. fp32 centroid -> bf16 hi + bf16 lo, rows padded to Mpad with zeros
+// ---------------------------------------------------------------------------------------------
+__global__ void split_centroid_kernel(const float* __restrict__ centroid, int M, int Mpad, int64_t n_rows_padded,
+                                      __nv_bfloat16* __restrict__ chi, __nv_bfloat16* __restrict__ clo) {
+  // one thread per 4 elements
+  const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+  const int64_t row = t / (kHeadDim / 4);
+  const int c4 = static_cast<int>(t % (kHeadDim / 4));
+  if (row >= n_rows_padded) return;
+  const int64_t hd = row / Mpad;
+  const int b = static_cast<int>(row % Mpad);
+  float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+  if (b < M) v = *reinterpret_cast<const float4*>(centroid + (hd * M + b) * kHeadDim + c4 * 4);
+  const __nv_bfloat16 h0 = __float2bfloat16_rn(v.x), h1 = __float2bfloat16_rn(v.y);
+  const __nv_bfloat16 h2 = __float2bfloat16_rn(v.z), h3 = __float2bfloat16_rn(v.w);
+  const float l0 = v.x - __bfloat162float(h0), l1 = v.y - __bfloat162float(h1);
+  const float l2 = v.z - __bfloat162float(h2), l3 = v.w - __bfloat162float(h3);
+  uint2 hi, lo;
+  hi.x = static_cast<uint32_t>(__bfloat16_as_ushort(h0)) | (static_cast<uint32_t>(__bfloat16_as_ushort(h1)) << 16);
+  hi.y = static_cast<uint32_t>(__bfloat16_as_ushort(h2)) | (static_cast<uint32_t>(__bfloat16_as_ushort(h3)) << 16);
+  lo.x = pack_bf16(l0, l1);
+  lo.y = pack_bf16(l2, l3);
+  *reinterpret_cast<uint2*>(chi + row * kHeadDim + c4 * 4) = hi;
+  *reinterpret_cast<uint2*>(clo + row * kHeadDim + c4 * 4) = lo;
+}
+
+// ---------------------------------------------------------------------------------------------
+// 3. scoring + thresholds + union + pack, one CTA per (l, query head, query block)
+// ---------------------------------------------------------------------------------------------
+constexpr int kSelThreads = 256;
+constexpr int kSelTileRows = 128;  // centroid rows per tile
+
+struct SelectParams {
+  const __nv_bfloat16* Q; int64_t qsb, qst, qsh;
+  const __nv_bfloat16* chi; const __nv_bfloat16* clo; const float* g;
+  int M, Mpad, W, L, Hq, G;
+  float scale_log2, t_base, t_rescue;  // thresholds as log2(alpha)
+  int n_sink, n_local, n_recent;
+  uint32_t* mask; uint32_t* dbg_base; uint32_t* dbg_rescue;
+  unsigned int* counts;
+};
+
+template <int B>
+__global__ void __launch_bounds__(kSelThreads)
+select_kernel(const SelectParams p) {
+  constexpr int NT = B / 8;  // n-tiles (tokens) per warp row-slab
+  extern __shared__ __align__(1024) unsigned char smem[];
+  unsigned char* sQ = smem;                                  // B x 256 B
+  unsigned char* sChi = sQ + B * 256;                        // 128 x 256 B
+  unsigned char* sClo = sChi + kSelTileRows * 256;           // 128 x 256 B
+  float* sQn = reinterpret_cast<float*>(sClo + kSelTileRows * 256);  // B
+  float* sRed = sQn + B;                                     // 32
+  float* sLb = sRed + 32;                                    // n_tiles * 128
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+
+  // heavy query blocks (large i) first
+  const int per_i = p.L * p.Hq;
+  const int i = p.M - 1 - static_cast<int>(blockIdx.x / per_i);
+  const int rem = static_cast<int>(blockIdx.x % per_i);
+  const int l = rem / p.Hq, h = rem % p.Hq, hk = h / p.G;
+  const int Hkv = p.Hq / p.G;
+  const int n_tiles = i / kSelTileRows + 1;
+  float* sLr = sLb + n_tiles * kSelTileRows;
+
+  const __nv_bfloat16* qbase = p.Q + l * p.qsb + static_cast<int64_t>(i) * B * p.qst + h * p.qsh;
+  const int64_t crow0 = (static_cast<int64_t>(l) * Hkv + hk) * p.Mpad;
+
+  auto load_ctile = [&](int bt) {
+    for (int c = tid; c < kSelTileRows * 16; c += kSelThreads) {
+      const int row = c >> 4, chunk = c & 15;
+      const int64_t src = (crow0 + bt * kSelTileRows + row) * kHeadDim + chunk * 8;
+      cp_async16(smem_u32(sChi + tile_off(row, chunk)), p.chi + src);
+      cp_async16(smem_u32(sClo + tile_off(row, chunk)), p.clo + src);
+    }
+  };
+
+  for (int c = tid; c < B * 16; c += kSelThreads) {
+    const int row = c >> 4, chunk = c & 15;
+    cp_async16(smem_u32(sQ + tile_off(row, chunk)), qbase + static_cast<int64_t>(row) * p.qst + chunk * 8);
+  }
+  load_ctile(0);
+  cp_async_commit();
+  cp_async_wait<0>();
+  __syncthreads();
+
+  // raw query norms ||q_t||_2
+  if (tid < B) {
+    float s = 0.f;
+#pragma unroll
+    for (int chunk = 0; chunk < 16; ++chunk) {
+      const uint4 v = *reinterpret_cast<const uint4*>(sQ + tile_off(tid, chunk));
+      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const float a = bf16lo(w[k]), c = bf16hi(w[k]);
+        s = fmaf(a, a, s);
+        s = fmaf(c, c, s);
+      }
+    }
+    sQn[tid] = sqrtf(s);
+  }
+  __syncthreads();
+
+  const int gq = lane >> 2, tq = lane & 3;
+  for (int bt = 0; bt < n_tiles; ++bt) {
+    float acc[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
+#pragma unroll
+    for (int k16 = 0; k16 < 8; ++k16) {
+      uint32_t ahi[4], alo[4];
+      const uint32_t aoff = tile_off(warp * 16 + (lane & 15), 2 * k16 + (lane >> 4));
+      ldmatrix_x4(ahi[0], ahi[1], ahi[2], ahi[3], smem_u32(sChi + aoff));
+      ldmatrix_x4(alo[0], alo[1], alo[2], alo[3], smem_u32(sClo + aoff));
+#pragma unroll
+      for (int ntp = 0; ntp < NT / 2; ++ntp) {
+        uint32_t b0, b1, b2, b3;
+        const int row = 16 * ntp + (lane & 7) + ((lane >> 4) << 3);
+        ldmatrix_x4(b0, b1, b2, b3, smem_u32(sQ + tile_off(row, 2 * k16 + ((lane >> 3) & 1))));
+        mma_bf16_16816(acc[2 * ntp], ahi, b0, b1);
+        mma_bf16_16816(acc[2 * ntp], alo, b0, b1);
+        mma_bf16_16816(acc[2 * ntp + 1], ahi, b2, b3);
+        mma_bf16_16816(acc[2 * ntp + 1], alo, b2, b3);
+      }
+    }
+    // per centroid row: log2-sum-exp2 over the block's tokens, both branches
+#pragma unroll
+    for (int rr = 0; rr < 2; ++rr) {
+      const int b = bt * kSelTileRows + warp * 16 + gq + rr * 8;
+      const float gb = p.g[crow0 + b];
+      float mb = -INFINITY, mr = -INFINITY;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const float2 qn = *reinterpret_cast<const float2*>(sQn + nt * 8 + tq * 2);
+        const float x0 = acc[nt][2 * rr] * p.scale_log2, x1 = acc[nt][2 * rr + 1] * p.scale_log2;
+        acc[nt][2 * rr] = x0; acc[nt][2 * rr + 1] = x1;
+        mb = fmaxf(mb, fmaxf(x0, x1));
+        mr = fmaxf(mr, fmaxf(fmaf(qn.x, gb, x0), fmaf(qn.y, gb, x1)));
+      }
+      mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, 1));
+      mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, 2));
+      mr = fmaxf(mr, __shfl_xor_sync(0xffffffffu, mr, 1));
+      mr = fmaxf(mr, __shfl_xor_sync(0xffffffffu, mr, 2));
+      float sb = 0.f, sr = 0.f;
+#pragma unroll
+      for (int nt = 0; nt < NT; ++nt) {
+        const float2 qn = *reinterpret_cast<const float2*>(sQn + nt * 8 + tq * 2);
+        const float x0 = acc[nt][2 * rr], x1 = acc[nt][2 * rr + 1];
+        sb += fast_exp2(x0 - mb) + fast_exp2(x1 - mb);
+        sr += fast_exp2(fmaf(qn.x, gb, x0) - mr) + fast_exp2(fmaf(qn.y, gb, x1) - mr);
+      }
+      sb += __shfl_xor_sync(0xffffffffu, sb, 1);
+      sb += __shfl_xor_sync(0xffffffffu, sb, 2);
+      sr += __shfl_xor_sync(0xffffffffu, sr, 1);
+      sr += __shfl_xor_sync(0xffffffffu, sr, 2);
+      if (tq == 0) {
+        const bool causal = b <= i;
+        sLb[b] = causal ? mb + fast_log2(sb) : -INFINITY;
+        sLr[b] = causal ? mr + fast_log2(sr) : -INFINITY;
+      }
+    }
+    __syncthreads();  // every warp is done with this centroid tile
+    if (bt + 1 < n_tiles) {
+      load_ctile(bt + 1);
+      cp_async_commit();
+      cp_async_wait<0>();
+      __syncthreads();
+    }
+  }
+
+  // row maxima over the causal candidates
+  float mxb = -INFINITY, mxr = -INFINITY;
+  for (int b = tid; b <= i; b += kSelThreads) { mxb = fmaxf(mxb, sLb[b]); mxr = fmaxf(mxr, sLr[b]); }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mxb = fmaxf(mxb, __shfl_xor_sync(0xffffffffu, mxb, o));
+    mxr = fmaxf(mxr, __shfl_xor_sync(0xffffffffu, mxr, o));
+  }
+  if (lane == 0) { sRed[warp] = mxb; sRed[8 + warp] = mxr; }
+  __syncthreads();
+  mxb = sRed[0]; mxr = sRed[8];
+#pragma unroll
+  for (int w = 1; w < kSelThreads / 32; ++w) { mxb = fmaxf(mxb, sRed[w]); mxr = fmaxf(mxr, sRed[8 + w]); }
+  const float thr_b = mxb + p.t_base, thr_r = mxr + p.t_rescue;
+
+  const int64_t mrow = ((static_cast<int64_t>(l) * p.Hq + h) * p.M + i) * p.W;
+  const bool all_forced = i >= p.M - p.n_recent;
+  unsigned int cnt = 0;
+  for (int w = warp; w < p.W; w += kSelThreads / 32) {
+    const int b = w * 32 + lane;
+    const bool valid = b <= i;
+    bool kb = false, kr = false, kf = false;
+    if (valid) {
+      kb = sLb[b] >= thr_b;
+      kr = sLr[b] >= thr_r;
+      kf = all_forced || b < p.n_sink || b > i - p.n_local;
+    }
+    const uint32_t wb = __ballot_sync(0xffffffffu, kb), wr = __ballot_sync(0xffffffffu, kr);
+    const uint32_t wf = __ballot_sync(0xffffffffu, kf);
+    if (lane == 0) {
+      const uint32_t word = wb | wr | wf;
+      p.mask[mrow + w] = word;
+      if (p.dbg_base) p.dbg_base[mrow + w] = wb;
+      if (p.dbg_rescue) p.dbg_rescue[mrow + w] = wr;
+      cnt += __popc(word);
+    }
+  }
+  if (lane == 0 && cnt) atomicAdd(p.counts + l * p.Hq + h, cnt);
+}
+
+__global__ void density_kernel(const unsigned int* __restrict__ counts, int n, int M, float* __restrict__ density) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t < n) {
+    const double pairs = 0.5 * static_cast<double>(M) * static_cast<double>(M + 1);
+    density[t] = static_cast<float>(static_cast<double>(counts[t]) / pairs);
+  }
+}
+
+template <int B>
+static rbs_status launch_select(const SelectParams& p, cudaStream_t s) {
+  const int n_tiles_max = (p.M + kSelTileRows - 1) / kSelTileRows;
+  const size_t smem = static_cast<size_t>(B) * 256 + 2 * kSelTileRows * 256 + (B + 32) * sizeof(float) +
+                      2 * static_cast<size_t>(n_tiles_max) * kSelTileRows * sizeof(float);
+  RBS_CUDA_OK(cudaFuncSetAttribute(select_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.M;
+  if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
+  select_kernel<B><<<static_cast<unsigned>(n_cta), kSelThreads, smem, s>>>(p);
+  RBS_CUDA_OK(cudaGetLastError());
+  return RBS_OK;
+}
+
+}  // namespace rbs
+
+extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats stats, float alpha_base,
+                                 float alpha_rescue, int n_sink, int n_local, int n_recent, uint32_t* mask,
+                                 float* density, uint32_t* dbg_base_mask, uint32_t* dbg_rescue_mask,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+  using namespace rbs;
+  rbs_status st = check_shape(shape);
+  if (st != RBS_OK) return st;
+  st = check_tensor(Q);
+  if (st != RBS_OK) return st;
+  if (!stats.centroid || !stats.radius || !stats.beta || !stats.rq || !mask || !density) return RBS_ERR_INVALID_ARG;
+  if (!(alpha_base > 0.f) || !(alpha_rescue > 0.f)) return RBS_ERR_INVALID_ARG;
+  if (n_sink < 0 || n_local < 0 || n_recent < 0) return RBS_ERR_INVALID_ARG;
+  Dims x = make_dims(*shape);
+  SelectWorkspace ws = select_workspace(x);
+  if (workspace == nullptr || workspace_bytes < ws.bytes) return RBS_ERR_WORKSPACE;
+  if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return RBS_ERR_WORKSPACE;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  unsigned char* wsp = static_cast<unsigned char*>(workspace);
+  __nv_bfloat16* chi = reinterpret_cast<__nv_bfloat16*>(wsp + ws.off_chi);
+  __nv_bfloat16* clo = reinterpret_cast<__nv_bfloat16*>(wsp + ws.off_clo);
+  float* g = reinterpret_cast<float*>(wsp + ws.off_g);
+  unsigned int* counts = reinterpret_cast<unsigned int*>(wsp + ws.off_counts);
+  const float scale_log2 = kLog2e / sqrtf(static_cast<float>(x.d));
+
+  int P = 1;
+  while (P < x.M) P <<= 1;
+  if (P < 2) P = 2;
+  const size_t coeff_smem = static_cast<size_t>(P) * sizeof(float);
+  RBS_CUDA_OK(cudaMemsetAsync(counts, 0, static_cast<size_t>(x.L) * x.Hq * sizeof(unsigned int), s));
+  rescue_coeff_kernel<<<x.L * x.Hkv, kCoeffThreads, coeff_smem, s>>>(stats.radius, x.M, P, scale_log2, stats.beta,
+                                                                     stats.rq, g, ws.Mpad);
+  RBS_CUDA_OK(cudaGetLastError());
+  const int64_t rows = static_cast<int64_t>(x.L) * x.Hkv * ws.Mpad;
+  const int64_t n_thr = rows * (kHeadDim / 4);
+  split_centroid_kernel<<<static_cast<unsigned>((n_thr + 255) / 256), 256, 0, s>>>(stats.centroid, x.M, ws.Mpad, rows, chi, clo);
+  RBS_CUDA_OK(cudaGetLastError());
+
+  SelectParams p;
+  p.Q = static_cast<const __nv_bfloat16*>(Q.ptr); p.qsb = Q.stride_batch; p.qst = Q.stride_token; p.qsh = Q.stride_head;
+  p.chi = chi; p.clo = clo; p.g = g;
+  p.M = x.M; p.Mpad = ws.Mpad; p.W = x.W; p.L = x.L; p.Hq = x.Hq; p.G = x.G;
+  p.scale_log2 = scale_log2; p.t_base = log2f(alpha_base); p.t_rescue = log2f(alpha_rescue);
+  p.n_sink = n_sink; p.n_local = n_local; p.n_recent = n_recent;
+  p.mask = mask; p.dbg_base = dbg_base_mask; p.dbg_rescue = dbg_rescue_mask; p.counts = counts;
+  st = (x.B == 128) ? launch_select<128>(p, s) : launch_select<64>(p, s);
+  if (st != RBS_OK) return st;
+  const int nh = x.L * x.Hq;
+  density_kernel<<<(nh + 127) / 128, 128, 0, s>>>(counts, nh, x.M, density);
+  RBS_CUDA_OK(cudaGetLastError());
+  return RBS_OK;
+}

@@ -1,0 +1,96 @@
+"""The C-ABI library loads without a GPU, exports every function include/rbs.h declares, and rejects bad
+arguments on the host before anything would be launched (so these calls are safe on a CPU-only box)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2609_20971_b200 import binding
+from paper_2609_20971_b200.binding import RbsShape, RbsStats, RbsTensor
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+OK, INVALID, UNSUPPORTED, WORKSPACE = 0, 1, 2, 3
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2609_20971_b200.build import build_library
+    build_library()
+    return binding.load_library()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "rbs.h")).read()
+    return re.findall(r"RBS_API\s+[\w\s\*]+?\b(rbs_\w+)\s*\(", text)
+
+
+def test_every_declared_symbol_is_exported(lib):
+    names = declared_functions()
+    assert {"rbs_block_stats", "rbs_select", "rbs_sparse_prefill", "rbs_workspace_bytes"} <= set(names)
+    for n in names:
+        assert hasattr(lib, n), n
+
+
+def test_status_strings_and_version(lib):
+    assert lib.rbs_status_string(0) == b"RBS_OK"
+    assert lib.rbs_status_string(2) == b"RBS_ERR_UNSUPPORTED"
+    assert b"sm_100a" in lib.rbs_version()
+
+
+def _t(ptr=0x1000, sb=0, st=128, sh=128):
+    return RbsTensor(ptr, sb, st, sh)
+
+
+def _stats(v=0x1000):
+    return RbsStats(v, v, v, v)
+
+
+def test_shape_checks_reject_before_launch(lib):
+    good = RbsShape(1, 1024, 4, 2, 128, 128)
+    cases = [
+        (RbsShape(1, 1024, 4, 2, 64, 128), UNSUPPORTED),    # head_dim
+        (RbsShape(1, 1024, 4, 2, 128, 32), UNSUPPORTED),    # block size
+        (RbsShape(1, 1000, 4, 2, 128, 128), UNSUPPORTED),   # ragged length
+        (RbsShape(1, 1024, 3, 2, 128, 128), UNSUPPORTED),   # heads not divisible
+        (RbsShape(0, 1024, 4, 2, 128, 128), INVALID),
+    ]
+    for shape, want in cases:
+        assert lib.rbs_block_stats(ctypes.byref(shape), _t(), _stats(), None) == want
+        assert lib.rbs_workspace_bytes(1, ctypes.byref(shape)) == 0
+    assert lib.rbs_block_stats(None, _t(), _stats(), None) == INVALID
+    assert lib.rbs_block_stats(ctypes.byref(good), _t(ptr=0), _stats(), None) == INVALID
+    assert lib.rbs_block_stats(ctypes.byref(good), _t(ptr=0x1008), _stats(), None) == INVALID   # misaligned
+    assert lib.rbs_block_stats(ctypes.byref(good), _t(st=100), _stats(), None) == INVALID       # stride % 8
+    assert lib.rbs_block_stats(ctypes.byref(good), _t(), _stats(0), None) == INVALID
+
+
+def test_select_argument_checks(lib):
+    good = RbsShape(1, 1024, 4, 2, 128, 128)
+    need = lib.rbs_workspace_bytes(1, ctypes.byref(good))
+    assert need > 0 and need % 256 == 0
+    p = ctypes.c_void_p(0x1000)
+
+    def call(alpha_b=0.22, alpha_r=0.18, sink=1, mask=p, ws=p, ws_bytes=need):
+        return lib.rbs_select(ctypes.byref(good), _t(), _stats(), alpha_b, alpha_r, sink, 1, 1, mask, p, None, None,
+                              ws, ws_bytes, None)
+    assert call(alpha_b=0.0) == INVALID
+    assert call(alpha_r=-1.0) == INVALID
+    assert call(sink=-1) == INVALID
+    assert call(mask=None) == INVALID
+    assert call(ws=None) == WORKSPACE
+    assert call(ws_bytes=need - 1) == WORKSPACE
+    assert call(ws=ctypes.c_void_p(0x1010)) == WORKSPACE          # not 256-byte aligned
+
+
+def test_prefill_argument_checks(lib):
+    good = RbsShape(1, 1024, 4, 2, 128, 128)
+    assert lib.rbs_sparse_prefill(ctypes.byref(good), _t(), _t(), _t(ptr=0), None, _t(), None, 0.0, None, 0, None) == INVALID
+    assert lib.rbs_sparse_prefill(ctypes.byref(good), _t(), _t(), _t(), None, _t(), None, -1.0, None, 0, None) == INVALID
+
+
+def test_binding_fails_loudly_when_library_is_missing(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(binding.RbsError):
+        binding.load_library()

@@ -1,0 +1,288 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the fp64 oracle on the same seeded inputs.
+
+Tolerances (from the build's target statement):
+  * integer / bit work (mask words, density bookkeeping): exact, except that a (query block, key block)
+    decision may differ from the oracle where the oracle's score is within 1e-3 (relative) of that
+    branch's threshold;
+  * attention output, bf16 inputs with fp32 accumulation: max-abs <= 2e-2 and mean-abs <= 2e-3;
+  * statistics (fp32 sums of <= 256 bf16 values): rtol 2e-5 against fp64.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import rbs_oracle as orc
+from paper_2609_20971_b200 import rbs_block_stats, rbs_select, rbs_sparse_prefill
+from paper_2609_20971_b200.synth import SynthConfig, make_inputs, paper_configs, to_f64
+
+pytestmark = pytest.mark.gpu
+
+MASK_MARGIN = 1e-3
+OUT_MAX_ABS = 2e-2
+OUT_MEAN_ABS = 2e-3
+
+
+def unpack_mask(mask: torch.Tensor, M: int) -> np.ndarray:
+    """[L, Hq, M, W] int32 words -> bool [L, Hq, M, M]."""
+    words = mask.cpu().numpy().view(np.uint32)
+    bits = (words[..., :, None] >> np.arange(32, dtype=np.uint32)) & 1
+    return bits.reshape(*words.shape[:-1], -1)[..., :M].astype(bool)
+
+
+def pack_mask(dense: np.ndarray) -> torch.Tensor:
+    """bool [L, Hq, M, M] -> int32 words [L, Hq, M, W]."""
+    L, H, M, _ = dense.shape
+    W = (M + 31) // 32
+    padded = np.zeros((L, H, M, W * 32), dtype=np.uint32)
+    padded[..., :M] = dense
+    words = (padded.reshape(L, H, M, W, 32) << np.arange(32, dtype=np.uint32)).sum(-1).astype(np.uint32)
+    return torch.from_numpy(words.view(np.int32))
+
+
+CASES = {
+    # name: config.  Sizes span several 128-row centroid tiles with a ragged tail and both block sizes.
+    "tiny_iid": paper_configs()["tiny_iid"],
+    "tiny": paper_configs()["tiny"],
+    "ragged_b64": SynthConfig("ragged_b64", N=64 * 300, Hq=2, Hkv=1, B=64, sigma=(0.1, 1.0), seed=31),
+    "gqa_b128": SynthConfig("gqa_b128", L=2, N=128 * 150, Hq=4, Hkv=2, B=128, sigma=(0.1, 1.0), seed=32,
+                            n_sink=2, n_local=3, n_recent=2),
+    "lognormal_b128": SynthConfig("lognormal_b128", N=128 * 40, Hq=2, Hkv=2, B=128, sigma=0.5, sigma_ln=0.5,
+                                  p_needle=0.05, seed=33),
+}
+
+
+@pytest.fixture(scope="module", params=list(CASES))
+def case(request):
+    cfg = CASES[request.param]
+    Q, K, V = make_inputs(cfg)
+    dev = torch.device("cuda:0")
+    Qg, Kg, Vg = Q.to(dev), K.to(dev), V.to(dev)
+    stats = rbs_block_stats(Kg, cfg.B)
+    mask, density, mb, mr = rbs_select(Qg, stats, cfg.B, cfg.alpha_base, cfg.alpha_rescue,
+                                       cfg.n_sink, cfg.n_local, cfg.n_recent, debug=True)
+    torch.cuda.synchronize()
+    Q64, K64 = to_f64(Q), to_f64(K)
+    ref = orc.select_all(Q64, K64, cfg.B, cfg.alpha_base, cfg.alpha_rescue, cfg.n_sink, cfg.n_local, cfg.n_recent)
+    return dict(cfg=cfg, Q=Q, K=K, V=V, Qg=Qg, Kg=Kg, Vg=Vg, stats=stats, mask=mask, density=density,
+                mb=mb, mr=mr, ref=ref, Q64=Q64, K64=K64, V64=to_f64(V))
+
+
+def test_block_stats_parity(case):
+    st, ref = case["stats"], case["ref"]
+    c = st.centroid.cpu().numpy().astype(np.float64)
+    r = st.radius.cpu().numpy().astype(np.float64)
+    assert np.allclose(c, ref.centroid, rtol=2e-5, atol=2e-6)
+    assert np.allclose(r, ref.radius, rtol=2e-5)
+
+
+def test_rescue_coefficient_parity(case):
+    st, ref = case["stats"], case["ref"]
+    assert np.allclose(st.rq.cpu().numpy(), ref.rq, rtol=5e-5)
+    assert np.allclose(st.beta.cpu().numpy(), ref.beta, atol=2e-4)
+    # plateaus are exact: beta == 0 at or below the median radius, == 1 at or above the 0.9 quantile
+    beta = st.beta.cpu().numpy()
+    lo, hi = ref.rq[..., 0:1], ref.rq[..., 1:2]
+    assert np.all(beta[ref.radius < lo * (1 - 1e-4)] == 0) and np.all(beta[ref.radius > hi * (1 + 1e-4)] == 1)
+
+
+def test_mask_parity(case):
+    cfg, ref = case["cfg"], case["ref"]
+    M = cfg.M
+    final = unpack_mask(case["mask"], M)
+    base = unpack_mask(case["mb"], M)
+    rescue = unpack_mask(case["mr"], M)
+    n_mismatch = 0
+    for l in range(cfg.L):
+        for h in range(cfg.Hq):
+            s = ref.selection[l][h]
+            near_b = s.margin_base <= MASK_MARGIN
+            near_r = s.margin_rescue <= MASK_MARGIN
+            assert not ((base[l, h] != s.base) & ~near_b).any()
+            assert not ((rescue[l, h] != s.rescue) & ~near_r).any()
+            bad = (final[l, h] != s.final) & ~(near_b | near_r)
+            assert not bad.any()
+            n_mismatch += int((final[l, h] != s.final).sum())
+            # the union is exact on the GPU's own branch masks, forced blocks always present, nothing above the diagonal
+            assert np.array_equal(final[l, h], base[l, h] | rescue[l, h] | s.forced)
+            assert not np.triu(final[l, h], 1).any()
+    pairs = M * (M + 1) // 2
+    assert n_mismatch <= max(2, int(2e-3 * pairs * cfg.L * cfg.Hq))   # near-threshold blocks are rare
+
+
+def test_density_parity(case):
+    cfg, ref = case["cfg"], case["ref"]
+    M = cfg.M
+    final = unpack_mask(case["mask"], M)
+    dens = case["density"].cpu().numpy()
+    pairs = M * (M + 1) // 2
+    for l in range(cfg.L):
+        for h in range(cfg.Hq):
+            assert dens[l, h] == np.float32(final[l, h].sum() / pairs)         # exact bookkeeping
+            allowed = ((ref.selection[l][h].margin_base <= MASK_MARGIN) |
+                       (ref.selection[l][h].margin_rescue <= MASK_MARGIN)).sum()
+            assert abs(dens[l, h] - ref.density[l, h]) <= (allowed + 0.5) / pairs
+
+
+def _check_output(O_gpu, O_ref):
+    err = np.abs(O_gpu - O_ref)
+    assert err.max() <= OUT_MAX_ABS, err.max()
+    assert err.mean() <= OUT_MEAN_ABS, err.mean()
+
+
+def _rows_to_check(cfg, n=12, seed=0):
+    M = cfg.M
+    rows = {0, 1, M - 1, M // 2}
+    rng = np.random.default_rng(seed)
+    rows |= {int(x) for x in rng.integers(0, M, size=n)}
+    return sorted(r for r in rows if 0 <= r < M)
+
+
+def test_sparse_attention_parity(case):
+    cfg = case["cfg"]
+    M, B, G = cfg.M, cfg.B, cfg.Hq // cfg.Hkv
+    O, lse = rbs_sparse_prefill(case["Qg"], case["Kg"], case["Vg"], case["mask"], B, return_lse=True)
+    torch.cuda.synchronize()
+    O = O.float().cpu().numpy().astype(np.float64)
+    lse = lse.cpu().numpy().astype(np.float64)
+    final = unpack_mask(case["mask"], M)     # the oracle attends over the mask the GPU kernel was given
+    every_row = M <= 64
+    for l in range(cfg.L):
+        for h in range(cfg.Hq):
+            hk = h // G
+            rows = range(M) if every_row else _rows_to_check(cfg, seed=l * 131 + h)
+            got, want, got_lse, want_lse = [], [], [], []
+            for i in rows:
+                o_ref, lse_ref = orc.masked_attention_block(case["Q64"][l, :, h], case["K64"][l, :, hk],
+                                                            case["V64"][l, :, hk], final[l, h, i], i, B)
+                want.append(o_ref); want_lse.append(lse_ref)
+                got.append(O[l, i * B:(i + 1) * B, h]); got_lse.append(lse[l, h, i * B:(i + 1) * B])
+            _check_output(np.concatenate(got), np.concatenate(want))
+            assert np.allclose(np.concatenate(got_lse), np.concatenate(want_lse), atol=2e-3, rtol=1e-4)
+
+
+def test_dense_attention_parity(case):
+    cfg = case["cfg"]
+    if cfg.N > 8192:
+        pytest.skip("dense oracle rows are checked on the small cases; large cases check sampled rows below")
+    B, G = cfg.B, cfg.Hq // cfg.Hkv
+    O = rbs_sparse_prefill(case["Qg"], case["Kg"], case["Vg"], None, B)
+    torch.cuda.synchronize()
+    O = O.float().cpu().numpy().astype(np.float64)
+    for l in range(cfg.L):
+        for h in range(cfg.Hq):
+            ref, _ = orc.dense_causal_attention(case["Q64"][l, :, h], case["K64"][l, :, h // G], case["V64"][l, :, h // G])
+            _check_output(O[l, :, h], ref)
+
+
+def test_dense_attention_sampled_rows(case):
+    cfg = case["cfg"]
+    if cfg.N <= 8192:
+        pytest.skip("covered in full by test_dense_attention_parity")
+    M, B, G = cfg.M, cfg.B, cfg.Hq // cfg.Hkv
+    O = rbs_sparse_prefill(case["Qg"], case["Kg"], case["Vg"], None, B)
+    torch.cuda.synchronize()
+    O = O.float().cpu().numpy().astype(np.float64)
+    full = np.ones(M, dtype=bool)
+    l, h = cfg.L - 1, cfg.Hq - 1
+    got, want = [], []
+    for i in (0, 1, M // 3, M - 1):
+        o_ref, _ = orc.masked_attention_block(case["Q64"][l, :, h], case["K64"][l, :, h // G], case["V64"][l, :, h // G], full, i, B)
+        want.append(o_ref); got.append(O[l, i * B:(i + 1) * B, h])
+    _check_output(np.concatenate(got), np.concatenate(want))
+
+
+# ------------------------------------------------------------------------------------------ edge cases
+def _small(B=64, M=5, Hq=2, Hkv=1, seed=40):
+    cfg = SynthConfig("edge", N=B * M, Hq=Hq, Hkv=Hkv, B=B, sigma=0.4, seed=seed)
+    Q, K, V = make_inputs(cfg)
+    return cfg, Q, K, V
+
+
+@pytest.mark.parametrize("B", [64, 128])
+def test_single_block_sequence(B):
+    cfg, Q, K, V = _small(B=B, M=1)
+    Qg, Kg, Vg = Q.cuda(), K.cuda(), V.cuda()
+    stats = rbs_block_stats(Kg, B)
+    mask, dens = rbs_select(Qg, stats, B)
+    assert unpack_mask(mask, 1).all() and np.all(dens.cpu().numpy() == 1.0)
+    assert np.all(stats.beta.cpu().numpy() == 0)            # one radius: degenerate quantiles
+    O = rbs_sparse_prefill(Qg, Kg, Vg, mask, B).float().cpu().numpy()
+    for h in range(cfg.Hq):
+        ref, _ = orc.dense_causal_attention(to_f64(Q)[0, :, h], to_f64(K)[0, :, 0], to_f64(V)[0, :, 0])
+        _check_output(O[0, :, h], ref)
+
+
+def test_hand_built_mask_empty_rows_and_bits_above_diagonal():
+    cfg, Q, K, V = _small(B=64, M=6)
+    M, B = cfg.M, cfg.B
+    dense = np.zeros((1, cfg.Hq, M, M), dtype=bool)
+    dense[0, 0] = np.tril(np.random.default_rng(1).random((M, M)) < 0.5)
+    dense[0, 0, 2, :] = False                     # an empty row
+    dense[0, 0, 3, :] = False
+    dense[0, 0, 3, 3] = True                      # diagonal only
+    dense[0, 1] = np.tril(np.ones((M, M), bool))
+    given = dense.copy()
+    given[0, 1, 1, 4] = True                      # bits with b > i must be ignored
+    given[0, 0, 2, 5] = True
+    mask = pack_mask(given).cuda()
+    O, lse = rbs_sparse_prefill(Q.cuda(), K.cuda(), V.cuda(), mask, B, return_lse=True)
+    O = O.float().cpu().numpy().astype(np.float64)
+    lse = lse.cpu().numpy()
+    for h in range(cfg.Hq):
+        for i in range(M):
+            ref, lref = orc.masked_attention_block(to_f64(Q)[0, :, h], to_f64(K)[0, :, 0], to_f64(V)[0, :, 0], dense[0, h, i], i, B)
+            _check_output(O[0, i * B:(i + 1) * B, h], ref)
+            if not dense[0, h, i].any():
+                assert not O[0, i * B:(i + 1) * B, h].any() and np.all(np.isneginf(lse[0, h, i * B:(i + 1) * B]))
+
+
+def test_branch_disable_and_degenerate_radii():
+    cfg, Q, K, V = _small(B=64, M=40, seed=41)
+    Qg, Kg = Q.cuda(), K.cuda()
+    stats = rbs_block_stats(Kg, cfg.B)
+    Q64, K64 = to_f64(Q), to_f64(K)
+    # rescue branch disabled (alpha > 1): final == base-branch mask, no forced blocks
+    mask, _, mb, mr = rbs_select(Qg, stats, cfg.B, 0.22, 2.0, 0, 0, 0, debug=True)
+    assert torch.equal(mask, mb) and not mr.any()
+    ref = orc.select_all(Q64, K64, cfg.B, 0.22, 2.0, 0, 0, 0)
+    for h in range(cfg.Hq):
+        s = ref.selection[0][h]
+        assert not ((unpack_mask(mask, cfg.M)[0, h] != s.final) & (s.margin_base > MASK_MARGIN)).any()
+    # both disabled: forced blocks only, density closed form 1 + 2 (M - 2) + M over M (M + 1) / 2
+    mask, dens = rbs_select(Qg, stats, cfg.B, 1.5, 1.5, 1, 1, 1)
+    M = cfg.M
+    assert np.allclose(dens.cpu().numpy(), (1 + 2 * (M - 2) + M) / (M * (M + 1) / 2))
+    # equal radii => beta == 0 => both branches score identically
+    stats.radius.fill_(3.0)
+    mask, _, mb, mr = rbs_select(Qg, stats, cfg.B, 0.2, 0.2, 0, 0, 0, debug=True)
+    assert not stats.beta.any() and torch.equal(mb, mr)
+
+
+def test_strided_views_of_a_packed_qkv_buffer():
+    cfg, Q, K, V = _small(B=128, M=9, Hq=4, Hkv=2, seed=42)
+    L, N, d = 1, cfg.N, cfg.d
+    packed = torch.empty(L, N, cfg.Hq + 2 * cfg.Hkv, d, dtype=torch.bfloat16, device="cuda")
+    packed[:, :, :cfg.Hq] = Q.cuda()
+    packed[:, :, cfg.Hq:cfg.Hq + cfg.Hkv] = K.cuda()
+    packed[:, :, cfg.Hq + cfg.Hkv:] = V.cuda()
+    Qv, Kv, Vv = packed[:, :, :cfg.Hq], packed[:, :, cfg.Hq:cfg.Hq + cfg.Hkv], packed[:, :, cfg.Hq + cfg.Hkv:]
+    s1 = rbs_block_stats(Kv, cfg.B)
+    s2 = rbs_block_stats(K.cuda(), cfg.B)
+    assert torch.equal(s1.centroid, s2.centroid) and torch.equal(s1.radius, s2.radius)
+    m1, d1 = rbs_select(Qv, s1, cfg.B)
+    m2, d2 = rbs_select(Q.cuda(), s2, cfg.B)
+    assert torch.equal(m1, m2) and torch.equal(d1, d2)
+    o1 = rbs_sparse_prefill(Qv, Kv, Vv, m1, cfg.B)
+    o2 = rbs_sparse_prefill(Q.cuda(), K.cuda(), V.cuda(), m2, cfg.B)
+    assert torch.equal(o1, o2)
+
+
+def test_select_is_deterministic_and_reusable_workspace():
+    cfg, Q, K, V = _small(B=64, M=33, seed=43)
+    Qg, Kg = Q.cuda(), K.cuda()
+    stats = rbs_block_stats(Kg, cfg.B)
+    m1, d1 = rbs_select(Qg, stats, cfg.B)
+    m2, d2 = rbs_select(Qg, stats, cfg.B)
+    assert torch.equal(m1, m2) and torch.equal(d1, d2)
