@@ -126,6 +126,16 @@ RBS_API rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, rbs_
                               const uint32_t* mask, rbs_tensor O, float* lse, float softmax_scale,
                               void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * Kernels that wait on hardware barriers (TMA arrival, tensor-core completion) give every wait an
+ * iteration limit.  A wait that runs out records a non-zero code in a device-side status word, lets the
+ * kernel drain and return, and leaves the CUDA context usable; outputs of that launch are then
+ * undefined.  This call synchronises `stream`, reads the word into *code_out (nullable) and, if
+ * `clear` is non-zero, resets it.  Returns RBS_OK when the word is 0, RBS_ERR_TIMEOUT otherwise.
+ * (No counterpart in the paper: an operational check.)
+ */
+RBS_API rbs_status rbs_device_status(void* stream, unsigned int* code_out, int clear);
+
 /* Human-readable name of a status code (static storage, never NULL). */
 RBS_API const char* rbs_status_string(rbs_status status);
 

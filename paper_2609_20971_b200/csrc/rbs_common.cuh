@@ -7,6 +7,8 @@
 
 #include "rbs.h"
 
+struct CUtensorMap_st;
+
 namespace rbs {
 
 constexpr int kHeadDim = 128;
@@ -38,6 +40,14 @@ struct SelectWorkspace {
   int Mpad;  // centroid rows per (l, hk) in the bf16 copies, multiple of 128
 };
 SelectWorkspace select_workspace(const Dims& x);
+
+// TMA tensor map over a bf16 [L][N][H][d] tensor with arbitrary (16-byte aligned) strides; box = box_d x box_t.
+rbs_status make_tmap_lthd(::CUtensorMap_st* out, const void* ptr, int L, int N, int H, int d, int64_t sb, int64_t st,
+                          int64_t sh, int box_d, int box_t, bool swizzle128);
+rbs_status make_tmap_2d(::CUtensorMap_st* out, const void* ptr, int64_t rows, int cols, int box_cols, int box_rows);
+int sm_count();
+// Device address of the status word that bounded waits report to (nullptr if it cannot be obtained).
+unsigned int* device_status_ptr();
 
 #define RBS_CUDA_OK(expr)                               \
   do {                                                  \

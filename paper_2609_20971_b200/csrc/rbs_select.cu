@@ -8,6 +8,7 @@
 // Scores are kept per block as log2-sum-exp2, L = log2 sum_t 2^(z_t); the relative threshold
 // S >= alpha max S becomes L >= log2(alpha) + max L (the common shift of Eq. block_aggregation cancels).
 #include "rbs_common.cuh"
+#include "rbs_sm100.cuh"
 
 namespace rbs {
 
@@ -275,6 +276,217 @@ select_kernel(const SelectParams p) {
   if (lane == 0 && cnt) atomicAdd(p.counts + l * p.Hq + h, cnt);
 }
 
+// ---------------------------------------------------------------------------------------------
+// 3b. the same scoring on the 5th-generation tensor cores.
+//   D[128 centroids x B tokens] (fp32, tensor memory) = C_hi . Q_i^T + C_lo . Q_i^T, 16 tcgen05.mma per tile.
+//   One TMEM lane = one centroid, so the aggregation over the block's tokens is a per-thread loop over
+//   the accumulator row: no cross-thread reduction at all.
+// Warp roles: warps 0-3 and 4-7 = two epilogue groups (tile parity), warp 8 = TMA producer,
+// warp 9 = MMA issuer and TMEM owner.
+// ---------------------------------------------------------------------------------------------
+constexpr int kTcThreads = 320;
+constexpr int kTcStages = 2;
+
+template <int B>
+__global__ void __launch_bounds__(kTcThreads, 1)
+select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmChi,
+                 const __grid_constant__ CUtensorMap tmClo, const SelectParams p, unsigned int* status) {
+  constexpr uint32_t kPanelC = 128 * 128;          // one 64-column panel of a 128-row centroid tile
+  constexpr uint32_t kStage = 4 * kPanelC;         // hi panels 0,1 then lo panels 0,1
+  constexpr uint32_t kPanelQ = B * 128;
+  constexpr uint32_t kIdesc = idesc_bf16_f32(128, B, false);
+  extern __shared__ __align__(1024) unsigned char smem[];
+  unsigned char* sC = smem;                                        // kTcStages x 64 KB
+  unsigned char* sQ = sC + kTcStages * kStage;                     // 2 panels
+  float* sQn = reinterpret_cast<float*>(sQ + 2 * kPanelQ);         // B
+  float* sRed = sQn + B;                                           // 32
+  float* sLb = sRed + 32;
+  __shared__ __align__(8) uint64_t bar_q, bar_cfull[kTcStages], bar_cempty[kTcStages], bar_tfull[2], bar_tempty[2];
+  __shared__ uint32_t s_tmem;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int per_i = p.L * p.Hq;
+  const int i = p.M - 1 - static_cast<int>(blockIdx.x / per_i);
+  const int rem = static_cast<int>(blockIdx.x % per_i);
+  const int l = rem / p.Hq, h = rem % p.Hq, hk = h / p.G;
+  const int Hkv = p.Hq / p.G;
+  const int n_tiles = i / 128 + 1;
+  float* sLr = sLb + n_tiles * 128;
+  const int crow0 = static_cast<int>((static_cast<int64_t>(l) * Hkv + hk) * p.Mpad);
+
+  if (tid == 0) {
+    mbar_init(smem_u32(&bar_q), 1);
+    for (int s = 0; s < kTcStages; ++s) { mbar_init(smem_u32(&bar_cfull[s]), 1); mbar_init(smem_u32(&bar_cempty[s]), 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bar_tfull[s]), 1); mbar_init(smem_u32(&bar_tempty[s]), 4); }
+    mbar_fence_init();
+  }
+  if (warp == 9) tmem_alloc(smem_u32(&s_tmem), 2 * B);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = s_tmem;
+
+  if (warp == 8) {
+    // ------------------------------- TMA producer -------------------------------
+    if (lane == 0) {
+      tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmChi); tma_prefetch_desc(&tmClo);
+      mbar_arrive_expect_tx(smem_u32(&bar_q), 2 * kPanelQ);
+      tma_load_4d(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, i * B, l);
+      tma_load_4d(smem_u32(sQ + kPanelQ), &tmQ, smem_u32(&bar_q), 64, h, i * B, l);
+      for (int bt = 0; bt < n_tiles; ++bt) {
+        const int s = bt % kTcStages, use = bt / kTcStages;
+        if (use > 0 && !mbar_wait(smem_u32(&bar_cempty[s]), (use - 1) & 1, status, kWaitStageFree)) break;
+        const uint32_t full = smem_u32(&bar_cfull[s]);
+        const uint32_t dst = smem_u32(sC + s * kStage);
+        mbar_arrive_expect_tx(full, kStage);
+        tma_load_2d(dst, &tmChi, full, 0, crow0 + bt * 128);
+        tma_load_2d(dst + kPanelC, &tmChi, full, 64, crow0 + bt * 128);
+        tma_load_2d(dst + 2 * kPanelC, &tmClo, full, 0, crow0 + bt * 128);
+        tma_load_2d(dst + 3 * kPanelC, &tmClo, full, 64, crow0 + bt * 128);
+      }
+    }
+  } else if (warp == 9) {
+    // ------------------------------- MMA issuer -------------------------------
+    if (lane == 0) {
+      bool ok = mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
+      for (int bt = 0; ok && bt < n_tiles; ++bt) {
+        const int s = bt % kTcStages, buf = bt & 1;
+        ok = mbar_wait(smem_u32(&bar_cfull[s]), (bt / kTcStages) & 1, status, kWaitTmaFull);
+        if (ok && bt >= 2) ok = mbar_wait(smem_u32(&bar_tempty[buf]), ((bt >> 1) - 1) & 1, status, kWaitTmemFree);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + buf * B;
+        const uint32_t cbase = smem_u32(sC + s * kStage);
+        const uint32_t qbase = smem_u32(sQ);
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+#pragma unroll
+          for (int k16 = 0; k16 < 8; ++k16) {
+            const uint64_t adesc = smem_desc_sw128(cbase + (2 * half + (k16 >> 2)) * kPanelC + (k16 & 3) * 32, 16, 1024);
+            const uint64_t bdesc = smem_desc_sw128(qbase + (k16 >> 2) * kPanelQ + (k16 & 3) * 32, 16, 1024);
+            mma_ss(d_tmem, adesc, bdesc, kIdesc, (half | k16) != 0);
+          }
+        }
+        mma_commit(smem_u32(&bar_cempty[s]));
+        mma_commit(smem_u32(&bar_tfull[buf]));
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------- epilogue groups -------------------------------
+    const int grp = warp >> 2;                       // tile parity handled by this group
+    const int row = (warp & 3) * 32 + lane;          // TMEM lane = centroid row inside the tile
+    bool ok = mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
+    // raw query norms (both groups compute the half they own; B <= 128 tokens, 256 epilogue threads)
+    if (ok && tid < B) {
+      float s2 = 0.f;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        const uint4 v = *reinterpret_cast<const uint4*>(sQ + (c >> 3) * kPanelQ + tid * 128 + (((c & 7) ^ (tid & 7)) << 4));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const float a = bf16lo(w[k]), c2 = bf16hi(w[k]);
+          s2 = fmaf(a, a, s2);
+          s2 = fmaf(c2, c2, s2);
+        }
+      }
+      sQn[tid] = sqrtf(s2);
+    }
+    asm volatile("bar.sync 1, 256;" ::: "memory");   // the eight epilogue warps
+    for (int bt = grp; ok && bt < n_tiles; bt += 2) {
+      ok = mbar_wait(smem_u32(&bar_tfull[grp]), (bt >> 1) & 1, status, kWaitMmaDone);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const int b = bt * 128 + row;
+      const float gb = p.g[crow0 + b];
+      const uint32_t taddr = tmem_base + grp * B + (static_cast<uint32_t>((warp & 3) * 32) << 16);
+      float mb = -INFINITY, mr = -INFINITY;
+#pragma unroll
+      for (int c0 = 0; c0 < B; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + c0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          const float4 qn = *reinterpret_cast<const float4*>(sQn + c0 + j);
+          const float x0 = __uint_as_float(r[j]) * p.scale_log2, x1 = __uint_as_float(r[j + 1]) * p.scale_log2;
+          const float x2 = __uint_as_float(r[j + 2]) * p.scale_log2, x3 = __uint_as_float(r[j + 3]) * p.scale_log2;
+          mb = fmaxf(mb, fmaxf(fmaxf(x0, x1), fmaxf(x2, x3)));
+          mr = fmaxf(mr, fmaxf(fmaxf(fmaf(qn.x, gb, x0), fmaf(qn.y, gb, x1)), fmaxf(fmaf(qn.z, gb, x2), fmaf(qn.w, gb, x3))));
+        }
+      }
+      float sb = 0.f, sr = 0.f;
+      const float nmb = -mb, nmr = -mr;
+#pragma unroll
+      for (int c0 = 0; c0 < B; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + c0, r);
+        tmem_wait_ld();
+        if (c0 + 32 >= B) {   // accumulator fully read: hand the TMEM buffer back to the MMA warp
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bar_tempty[grp]));
+        }
+#pragma unroll
+        for (int j = 0; j < 32; j += 4) {
+          const float4 qn = *reinterpret_cast<const float4*>(sQn + c0 + j);
+          const float x0 = __uint_as_float(r[j]) * p.scale_log2, x1 = __uint_as_float(r[j + 1]) * p.scale_log2;
+          const float x2 = __uint_as_float(r[j + 2]) * p.scale_log2, x3 = __uint_as_float(r[j + 3]) * p.scale_log2;
+          sb += fast_exp2(x0 + nmb) + fast_exp2(x1 + nmb) + fast_exp2(x2 + nmb) + fast_exp2(x3 + nmb);
+          sr += fast_exp2(fmaf(qn.x, gb, x0) + nmr) + fast_exp2(fmaf(qn.y, gb, x1) + nmr) +
+                fast_exp2(fmaf(qn.z, gb, x2) + nmr) + fast_exp2(fmaf(qn.w, gb, x3) + nmr);
+        }
+      }
+      const bool causal = b <= i;
+      sLb[b] = causal ? mb + fast_log2(sb) : -INFINITY;
+      sLr[b] = causal ? mr + fast_log2(sr) : -INFINITY;
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  if (warp == 9) tmem_dealloc(tmem_base, 2 * B);
+
+  // row maxima over the causal candidates, thresholds, forced blocks, union, pack (all ten warps)
+  float mxb = -INFINITY, mxr = -INFINITY;
+  for (int b = tid; b <= i; b += kTcThreads) { mxb = fmaxf(mxb, sLb[b]); mxr = fmaxf(mxr, sLr[b]); }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mxb = fmaxf(mxb, __shfl_xor_sync(0xffffffffu, mxb, o));
+    mxr = fmaxf(mxr, __shfl_xor_sync(0xffffffffu, mxr, o));
+  }
+  if (lane == 0) { sRed[warp] = mxb; sRed[16 + warp] = mxr; }
+  __syncthreads();
+  mxb = sRed[0]; mxr = sRed[16];
+#pragma unroll
+  for (int w = 1; w < kTcThreads / 32; ++w) { mxb = fmaxf(mxb, sRed[w]); mxr = fmaxf(mxr, sRed[16 + w]); }
+  const float thr_b = mxb + p.t_base, thr_r = mxr + p.t_rescue;
+  const int64_t mrow = ((static_cast<int64_t>(l) * p.Hq + h) * p.M + i) * p.W;
+  const bool all_forced = i >= p.M - p.n_recent;
+  unsigned int cnt = 0;
+  for (int w = warp; w < p.W; w += kTcThreads / 32) {
+    const int b = w * 32 + lane;
+    const bool valid = b <= i;
+    bool kb = false, kr = false, kf = false;
+    if (valid) {
+      kb = sLb[b] >= thr_b;
+      kr = sLr[b] >= thr_r;
+      kf = all_forced || b < p.n_sink || b > i - p.n_local;
+    }
+    const uint32_t wb = __ballot_sync(0xffffffffu, kb), wr = __ballot_sync(0xffffffffu, kr);
+    const uint32_t wf = __ballot_sync(0xffffffffu, kf);
+    if (lane == 0) {
+      const uint32_t word = wb | wr | wf;
+      p.mask[mrow + w] = word;
+      if (p.dbg_base) p.dbg_base[mrow + w] = wb;
+      if (p.dbg_rescue) p.dbg_rescue[mrow + w] = wr;
+      cnt += __popc(word);
+    }
+  }
+  if (lane == 0 && cnt) atomicAdd(p.counts + l * p.Hq + h, cnt);
+}
+
 __global__ void density_kernel(const unsigned int* __restrict__ counts, int n, int M, float* __restrict__ density) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t < n) {
@@ -296,7 +508,32 @@ static rbs_status launch_select(const SelectParams& p, cudaStream_t s) {
   return RBS_OK;
 }
 
+template <int B>
+static rbs_status launch_select_tc(const SelectParams& p, const rbs_tensor& Q, int N, cudaStream_t s) {
+  CUtensorMap tmQ, tmChi, tmClo;
+  rbs_status st = make_tmap_lthd(&tmQ, Q.ptr, p.L, N, p.Hq, kHeadDim, Q.stride_batch, Q.stride_token, Q.stride_head, 64, B, true);
+  if (st != RBS_OK) return st;
+  const int64_t rows = static_cast<int64_t>(p.L) * (p.Hq / p.G) * p.Mpad;
+  if ((st = make_tmap_2d(&tmChi, p.chi, rows, kHeadDim, 64, 128)) != RBS_OK) return st;
+  if ((st = make_tmap_2d(&tmClo, p.clo, rows, kHeadDim, 64, 128)) != RBS_OK) return st;
+  unsigned int* status = device_status_ptr();
+  if (status == nullptr) return RBS_ERR_CUDA;
+  const int n_tiles_max = (p.M + 127) / 128;
+  const size_t smem = static_cast<size_t>(kTcStages) * 4 * 128 * 128 + 2 * static_cast<size_t>(B) * 128 +
+                      (B + 32) * sizeof(float) + 2 * static_cast<size_t>(n_tiles_max) * 128 * sizeof(float);
+  auto kern = select_tc_kernel<B>;
+  RBS_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.M;
+  if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
+  kern<<<static_cast<unsigned>(n_cta), kTcThreads, smem, s>>>(tmQ, tmChi, tmClo, p, status);
+  RBS_CUDA_OK(cudaGetLastError());
+  return RBS_OK;
+}
+
 }  // namespace rbs
+
+static int g_select_variant = 1;  // 0: mma.sync, 1: tcgen05
+extern "C" __attribute__((visibility("default"))) void rbs_dev_set_select_variant(int v) { g_select_variant = v; }
 
 extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats stats, float alpha_base,
                                  float alpha_rescue, int n_sink, int n_local, int n_recent, uint32_t* mask,
@@ -342,7 +579,10 @@ extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats
   p.scale_log2 = scale_log2; p.t_base = log2f(alpha_base); p.t_rescue = log2f(alpha_rescue);
   p.n_sink = n_sink; p.n_local = n_local; p.n_recent = n_recent;
   p.mask = mask; p.dbg_base = dbg_base_mask; p.dbg_rescue = dbg_rescue_mask; p.counts = counts;
-  st = (x.B == 128) ? launch_select<128>(p, s) : launch_select<64>(p, s);
+  if (g_select_variant == 1)
+    st = (x.B == 128) ? launch_select_tc<128>(p, Q, x.N, s) : launch_select_tc<64>(p, Q, x.N, s);
+  else
+    st = (x.B == 128) ? launch_select<128>(p, s) : launch_select<64>(p, s);
   if (st != RBS_OK) return st;
   const int nh = x.L * x.Hq;
   density_kernel<<<(nh + 127) / 128, 128, 0, s>>>(counts, nh, x.M, density);

@@ -1,96 +1,136 @@
-// rbs_block_stats: one HBM stream over K.  Each CTA owns one (batch, KV head, key block) tile of
-// B rows x 128 bf16, holds it in registers, and produces the centroid and the radius from that single read.
+// rbs_block_stats: one HBM stream over K.  Each warp owns one (batch, KV head, key block) tile of
+// B rows x 128 bf16 at a time, brought into shared memory by TMA, and produces the centroid and the
+// radius from that single read of K.
 #include "rbs_common.cuh"
+#include "rbs_sm100.cuh"
 
 namespace rbs {
 
-constexpr int kStatsThreads = 256;
+// ---------------------------------------------------------------------------------------------
+// Every warp owns one shared-memory slot, fetches its own tiles with TMA
+// (two 128-byte-swizzled panels of 64 columns) and reduces them alone, so warps never wait for one
+// another.  Pass 1: lanes own 4 columns and walk the rows (column sums, no cross-lane traffic).
+// Pass 2: lanes own rows and walk the columns (row distances, no cross-lane traffic); the swizzle
+// keeps both access patterns free of bank conflicts.
+// ---------------------------------------------------------------------------------------------
+template <int B, int NW>
+__global__ void __launch_bounds__(NW * 32, 1)
+block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, int M, int Hkv,
+                        float* __restrict__ centroid, float* __restrict__ radius, unsigned int* status) {
+  constexpr uint32_t kPanel = B * 128;       // bytes of one 64-column panel
+  constexpr uint32_t kSlot = 2 * kPanel;
+  constexpr int RJ = B / 32;                  // rows per lane in pass 2
+  extern __shared__ __align__(1024) unsigned char smem[];
+  __shared__ __align__(8) uint64_t full_bar[NW];
 
-// Thread t owns 16-byte chunk (t % 16) of rows (t / 16) + 16 j, j < B / 16.
-template <int B>
-__global__ void __launch_bounds__(kStatsThreads)
-block_stats_kernel(const __nv_bfloat16* __restrict__ K, int64_t sb, int64_t st, int64_t sh, int M, int Hkv,
-                   float* __restrict__ centroid, float* __restrict__ radius) {
-  constexpr int R = B / 16;  // rows per thread
-  __shared__ float s_part[kStatsThreads / 32][kHeadDim];
-  __shared__ float s_max[kStatsThreads / 32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const uint32_t bar = smem_u32(&full_bar[warp]);
+  const uint32_t slot = smem_u32(smem) + warp * kSlot;
+  if (lane == 0) {
+    mbar_init(bar, 1);
+    mbar_fence_init();
+  }
+  __syncwarp();
 
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int chunk = tid & 15, r0 = tid >> 4;
-  // KV head fastest so that neighbouring CTAs read neighbouring 256-byte rows of the same tokens.
-  int idx = blockIdx.x;
-  const int hk = idx % Hkv; idx /= Hkv;
-  const int b = idx % M;
-  const int l = idx / M;
+  const int stride = gridDim.x * NW;
+  int t = warp * gridDim.x + blockIdx.x;
+  auto issue = [&](int tile) {
+    int idx = tile;
+    const int hk = idx % Hkv; idx /= Hkv;
+    const int b = idx % M;
+    const int l = idx / M;
+    mbar_arrive_expect_tx(bar, kSlot);
+    tma_load_4d(slot, &tmK, bar, 0, hk, b * B, l);
+    tma_load_4d(slot + kPanel, &tmK, bar, 64, hk, b * B, l);
+  };
+  if (lane == 0 && t < n_tiles) issue(t);
 
-  const __nv_bfloat16* base = K + l * sb + (static_cast<int64_t>(b) * B + r0) * st + hk * sh + chunk * 8;
-  uint4 v[R];
+  // pass-1 addressing: lane owns 8 bytes (4 columns): 16-byte chunk c16 = lane / 2, half = lane % 2
+  const int c16 = lane >> 1, cp = c16 & 7;
+  const uint32_t p1_base = slot + (c16 >> 3) * kPanel + (lane & 1) * 8;
+  uint32_t phase = 0;
+  for (; t < n_tiles; t += stride, phase ^= 1) {
+    if (!mbar_wait(bar, phase, status, kWaitTmaFull)) break;
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll 4
+    for (int r8 = 0; r8 < B; r8 += 8) {
 #pragma unroll
-  for (int j = 0; j < R; ++j) v[j] = __ldg(reinterpret_cast<const uint4*>(base + static_cast<int64_t>(16 * j) * st));
+      for (int rr = 0; rr < 8; ++rr) {
+        uint32_t lo, hi;
+        asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(lo), "=r"(hi)
+                     : "r"(p1_base + (r8 + rr) * 128 + ((cp ^ rr) << 4)));
+        a0 += bf16lo(lo); a1 += bf16hi(lo); a2 += bf16lo(hi); a3 += bf16hi(hi);
+      }
+    }
+    const float4 cen = make_float4(a0 * (1.0f / B), a1 * (1.0f / B), a2 * (1.0f / B), a3 * (1.0f / B));
+    int idx = t;
+    const int hk = idx % Hkv; idx /= Hkv;
+    const int b = idx % M;
+    const int l = idx / M;
+    const int64_t blk = (static_cast<int64_t>(l) * Hkv + hk) * M + b;
+    reinterpret_cast<float4*>(centroid + blk * kHeadDim)[lane] = cen;
 
-  float acc[8];
+    float q[RJ];
 #pragma unroll
-  for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+    for (int j = 0; j < RJ; ++j) q[j] = 0.f;
+    const uint32_t row_base = slot + lane * 128;
+    const int sw = lane & 7;
 #pragma unroll
-  for (int j = 0; j < R; ++j) {
-    acc[0] += bf16lo(v[j].x); acc[1] += bf16hi(v[j].x);
-    acc[2] += bf16lo(v[j].y); acc[3] += bf16hi(v[j].y);
-    acc[4] += bf16lo(v[j].z); acc[5] += bf16hi(v[j].z);
-    acc[6] += bf16lo(v[j].w); acc[7] += bf16hi(v[j].w);
+    for (int c = 0; c < 16; ++c) {
+      // centroid columns 8c..8c+7 live in lanes 2c and 2c+1
+      float4 ca, cb;
+      ca.x = __shfl_sync(0xffffffffu, cen.x, 2 * c); ca.y = __shfl_sync(0xffffffffu, cen.y, 2 * c);
+      ca.z = __shfl_sync(0xffffffffu, cen.z, 2 * c); ca.w = __shfl_sync(0xffffffffu, cen.w, 2 * c);
+      cb.x = __shfl_sync(0xffffffffu, cen.x, 2 * c + 1); cb.y = __shfl_sync(0xffffffffu, cen.y, 2 * c + 1);
+      cb.z = __shfl_sync(0xffffffffu, cen.z, 2 * c + 1); cb.w = __shfl_sync(0xffffffffu, cen.w, 2 * c + 1);
+      const uint32_t col = (c >> 3) * kPanel + (((c & 7) ^ sw) << 4);
+#pragma unroll
+      for (int j = 0; j < RJ; ++j) {
+        uint32_t x0, x1, x2, x3;
+        asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(x0), "=r"(x1), "=r"(x2), "=r"(x3)
+                     : "r"(row_base + j * 32 * 128 + col));
+        float d;
+        d = bf16lo(x0) - ca.x; q[j] = fmaf(d, d, q[j]);
+        d = bf16hi(x0) - ca.y; q[j] = fmaf(d, d, q[j]);
+        d = bf16lo(x1) - ca.z; q[j] = fmaf(d, d, q[j]);
+        d = bf16hi(x1) - ca.w; q[j] = fmaf(d, d, q[j]);
+        d = bf16lo(x2) - cb.x; q[j] = fmaf(d, d, q[j]);
+        d = bf16hi(x2) - cb.y; q[j] = fmaf(d, d, q[j]);
+        d = bf16lo(x3) - cb.z; q[j] = fmaf(d, d, q[j]);
+        d = bf16hi(x3) - cb.w; q[j] = fmaf(d, d, q[j]);
+      }
+    }
+    float rmax = q[0];
+#pragma unroll
+    for (int j = 1; j < RJ; ++j) rmax = fmaxf(rmax, q[j]);
+    __syncwarp();   // every lane is done reading the slot
+    if (lane == 0 && t + stride < n_tiles) {
+      fence_proxy_async_smem();
+      issue(t + stride);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, o));
+    if (lane == 0) radius[blk] = sqrtf(rmax);
   }
-#pragma unroll
-  for (int k = 0; k < 8; ++k) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], 16);
-  if (lane < 16) {
-    float4* p = reinterpret_cast<float4*>(&s_part[warp][chunk * 8]);
-    p[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-    p[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
-  }
-  __syncthreads();
-  float cen[8];
-#pragma unroll
-  for (int k = 0; k < 8; ++k) cen[k] = 0.f;
-#pragma unroll
-  for (int w = 0; w < kStatsThreads / 32; ++w) {
-    const float4* p = reinterpret_cast<const float4*>(&s_part[w][chunk * 8]);
-    float4 a = p[0], c = p[1];
-    cen[0] += a.x; cen[1] += a.y; cen[2] += a.z; cen[3] += a.w;
-    cen[4] += c.x; cen[5] += c.y; cen[6] += c.z; cen[7] += c.w;
-  }
-#pragma unroll
-  for (int k = 0; k < 8; ++k) cen[k] *= (1.0f / B);
-  const int64_t blk = (static_cast<int64_t>(l) * Hkv + hk) * M + b;
-  if (tid < 16) {
-    float4* out = reinterpret_cast<float4*>(centroid + blk * kHeadDim + chunk * 8);
-    out[0] = make_float4(cen[0], cen[1], cen[2], cen[3]);
-    out[1] = make_float4(cen[4], cen[5], cen[6], cen[7]);
-  }
+}
 
-  // radius^2 = max over rows of sum_j (k_j - c_j)^2, difference form
-  float rmax = 0.f;
-#pragma unroll
-  for (int j = 0; j < R; ++j) {
-    float d0 = bf16lo(v[j].x) - cen[0], d1 = bf16hi(v[j].x) - cen[1];
-    float d2 = bf16lo(v[j].y) - cen[2], d3 = bf16hi(v[j].y) - cen[3];
-    float d4 = bf16lo(v[j].z) - cen[4], d5 = bf16hi(v[j].z) - cen[5];
-    float d6 = bf16lo(v[j].w) - cen[6], d7 = bf16hi(v[j].w) - cen[7];
-    float s = d0 * d0;
-    s = fmaf(d1, d1, s); s = fmaf(d2, d2, s); s = fmaf(d3, d3, s);
-    s = fmaf(d4, d4, s); s = fmaf(d5, d5, s); s = fmaf(d6, d6, s); s = fmaf(d7, d7, s);
-    s += __shfl_xor_sync(0xffffffffu, s, 1);
-    s += __shfl_xor_sync(0xffffffffu, s, 2);
-    s += __shfl_xor_sync(0xffffffffu, s, 4);
-    s += __shfl_xor_sync(0xffffffffu, s, 8);
-    rmax = fmaxf(rmax, s);
-  }
-  rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, 16));
-  if (lane == 0) s_max[warp] = rmax;
-  __syncthreads();
-  if (tid == 0) {
-    float m = s_max[0];
-#pragma unroll
-    for (int w = 1; w < kStatsThreads / 32; ++w) m = fmaxf(m, s_max[w]);
-    radius[blk] = sqrtf(m);
-  }
+template <int B, int NW>
+static rbs_status launch_stats_warp(const rbs_tensor& K, const Dims& x, const rbs_stats& stats, cudaStream_t s) {
+  CUtensorMap tm;
+  rbs_status st = make_tmap_lthd(&tm, K.ptr, x.L, x.N, x.Hkv, x.d, K.stride_batch, K.stride_token, K.stride_head,
+                                 64, B, true);
+  if (st != RBS_OK) return st;
+  unsigned int* status = device_status_ptr();
+  if (status == nullptr) return RBS_ERR_CUDA;
+  const size_t smem = static_cast<size_t>(NW) * B * 256;
+  auto kern = block_stats_warp_kernel<B, NW>;
+  RBS_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  const long long n_tiles = static_cast<long long>(x.L) * x.Hkv * x.M;
+  long long want = (n_tiles + NW - 1) / NW;
+  const int grid = static_cast<int>(want < sm_count() ? want : sm_count());
+  kern<<<grid, NW * 32, smem, s>>>(tm, static_cast<int>(n_tiles), x.M, x.Hkv, stats.centroid, stats.radius, status);
+  RBS_CUDA_OK(cudaGetLastError());
+  return RBS_OK;
 }
 
 }  // namespace rbs
@@ -107,14 +147,5 @@ extern "C" rbs_status rbs_block_stats(const rbs_shape* shape, rbs_tensor K, rbs_
   const long long n_tiles = static_cast<long long>(x.L) * x.Hkv * x.M;
   if (n_tiles > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  const __nv_bfloat16* k = static_cast<const __nv_bfloat16*>(K.ptr);
-  dim3 grid(static_cast<unsigned>(n_tiles));
-  if (x.B == 128)
-    block_stats_kernel<128><<<grid, kStatsThreads, 0, s>>>(k, K.stride_batch, K.stride_token, K.stride_head, x.M, x.Hkv,
-                                                            stats.centroid, stats.radius);
-  else
-    block_stats_kernel<64><<<grid, kStatsThreads, 0, s>>>(k, K.stride_batch, K.stride_token, K.stride_head, x.M, x.Hkv,
-                                                           stats.centroid, stats.radius);
-  RBS_CUDA_OK(cudaGetLastError());
-  return RBS_OK;
+  return x.B == 128 ? launch_stats_warp<128, 7>(K, x, stats, s) : launch_stats_warp<64, 14>(K, x, stats, s);
 }
