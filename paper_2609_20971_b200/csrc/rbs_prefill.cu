@@ -2,6 +2,7 @@
 // the mask is NULL (Eq. 1).  One CTA per (batch, query head, query block); it walks the set bits of its
 // mask row, streams those K/V blocks through shared memory and keeps an online softmax in registers.
 #include "rbs_common.cuh"
+#include "rbs_sm100.cuh"
 
 namespace rbs {
 
@@ -209,6 +210,227 @@ prefill_mma_kernel(const PrefillParams p) {
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Tensor-core path for B = 128: TMA-fed, tcgen05.mma with the accumulators in tensor memory.
+//   S[128 q x 128 keys] = Q_i K_b^T          (both operands from shared memory, 8 MMAs of K = 16)
+//   O[128 q x 128 d]   += P V_b              (P from tensor memory, V_b from shared memory, 8 MMAs)
+// One CTA per (batch, query head, query block), two CTAs per SM so that one CTA's softmax overlaps the
+// other's matrix multiplies.  TMEM columns: [0,128) S, with P (bf16 pairs) written over [0,64) once a
+// thread has read its S row; [128,256) O.
+// Warps 0-3: softmax, one query row per thread (TMEM lane = row).  Warp 4: TMA producer.  Warp 5: MMA issuer.
+// The running row maximum is only raised when a block exceeds it by more than kRescaleSlack (log2 units);
+// P then stays below 2^kRescaleSlack and O is rescaled rarely.
+// ---------------------------------------------------------------------------------------------
+constexpr int kPfThreads = 192;
+constexpr float kRescaleSlack = 8.0f;
+
+__global__ void __launch_bounds__(kPfThreads, 2)
+prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                  const __grid_constant__ CUtensorMap tmV, const PrefillParams p, unsigned int* status) {
+  constexpr int B = 128;
+  constexpr uint32_t kPanel = B * 128;   // 16 KB: 128 rows x 64 bf16 columns
+  constexpr uint32_t kTile = 2 * kPanel;
+  constexpr uint32_t kIdescQK = idesc_bf16_f32(128, 128, false);
+  constexpr uint32_t kIdescPV = idesc_bf16_f32(128, 128, true);
+  extern __shared__ __align__(1024) unsigned char smem[];
+  unsigned char* sQ = smem;
+  unsigned char* sK = smem + kTile;
+  unsigned char* sV = smem + 2 * kTile;
+  __shared__ __align__(8) uint64_t bar_q, bar_kfull, bar_vfull, bar_s, bar_p, bar_pv;
+  __shared__ uint32_t s_tmem;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int per_i = p.L * p.Hq;
+  const int i = p.M - 1 - static_cast<int>(blockIdx.x / per_i);
+  const int rem = static_cast<int>(blockIdx.x % per_i);
+  const int l = rem / p.Hq, h = rem % p.Hq, hk = h / p.G;
+  const uint32_t* mrow = p.mask ? p.mask + ((static_cast<int64_t>(l) * p.Hq + h) * p.M + i) * p.W : nullptr;
+
+  if (tid == 0) {
+    mbar_init(smem_u32(&bar_q), 1);
+    mbar_init(smem_u32(&bar_kfull), 1);
+    mbar_init(smem_u32(&bar_vfull), 1);
+    mbar_init(smem_u32(&bar_s), 1);
+    mbar_init(smem_u32(&bar_p), 128);
+    mbar_init(smem_u32(&bar_pv), 1);
+    mbar_fence_init();
+  }
+  if (warp == 5) tmem_alloc(smem_u32(&s_tmem), 256);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_s = s_tmem, tmem_o = s_tmem + 128;
+
+  if (warp == 4) {
+    // ------------------------------- TMA producer -------------------------------
+    if (lane == 0) {
+      tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+      int b = next_block(mrow, -1, i);
+      if (b >= 0) {
+        mbar_arrive_expect_tx(smem_u32(&bar_q), kTile);
+        tma_load_4d(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, i * B, l);
+        tma_load_4d(smem_u32(sQ + kPanel), &tmQ, smem_u32(&bar_q), 64, h, i * B, l);
+      }
+      for (int j = 0; b >= 0; ++j, b = next_block(mrow, b, i)) {
+        if (j > 0 && !mbar_wait(smem_u32(&bar_s), (j - 1) & 1, status, kWaitStageFree)) break;   // S_{j-1} done: K free
+        mbar_arrive_expect_tx(smem_u32(&bar_kfull), kTile);
+        tma_load_4d(smem_u32(sK), &tmK, smem_u32(&bar_kfull), 0, hk, b * B, l);
+        tma_load_4d(smem_u32(sK + kPanel), &tmK, smem_u32(&bar_kfull), 64, hk, b * B, l);
+        if (j > 0 && !mbar_wait(smem_u32(&bar_pv), (j - 1) & 1, status, kWaitStageFree)) break;  // O_{j-1} done: V free
+        mbar_arrive_expect_tx(smem_u32(&bar_vfull), kTile);
+        tma_load_4d(smem_u32(sV), &tmV, smem_u32(&bar_vfull), 0, hk, b * B, l);
+        tma_load_4d(smem_u32(sV + kPanel), &tmV, smem_u32(&bar_vfull), 64, hk, b * B, l);
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------- MMA issuer -------------------------------
+    if (lane == 0) {
+      int b = next_block(mrow, -1, i);
+      bool ok = b < 0 || mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
+      const uint32_t qb = smem_u32(sQ), kb = smem_u32(sK), vb = smem_u32(sV);
+      for (int j = 0; ok && b >= 0; ++j, b = next_block(mrow, b, i)) {
+        const uint32_t ph = j & 1;
+        if (!(ok = mbar_wait(smem_u32(&bar_kfull), ph, status, kWaitTmaFull))) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int k16 = 0; k16 < 8; ++k16) {
+          const uint32_t off = (k16 >> 2) * kPanel + (k16 & 3) * 32;
+          mma_ss(tmem_s, smem_desc_sw128(qb + off, 16, 1024), smem_desc_sw128(kb + off, 16, 1024), kIdescQK, k16 != 0);
+        }
+        mma_commit(smem_u32(&bar_s));
+        if (!(ok = mbar_wait(smem_u32(&bar_p), ph, status, kWaitPReady))) break;
+        if (!(ok = mbar_wait(smem_u32(&bar_vfull), ph, status, kWaitTmaFull))) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int k16 = 0; k16 < 8; ++k16)
+          mma_ts(tmem_o, tmem_s + k16 * 8, smem_desc_sw128(vb + k16 * 2048, kPanel, 1024), kIdescPV, (j | k16) != 0);
+        mma_commit(smem_u32(&bar_pv));
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------- softmax: one query row per thread -------------------------------
+    const int row = warp * 32 + lane;
+    const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
+    float m_used = -INFINITY, l_sum = 0.f;   // m_used in log2 units of the scaled logits
+    int b = next_block(mrow, -1, i);
+    const bool any_block = b >= 0;
+    bool ok = true;
+    int j = 0;
+    for (; b >= 0; ++j, b = next_block(mrow, b, i)) {
+      if (!(ok = mbar_wait(smem_u32(&bar_s), j & 1, status, kWaitMmaDone))) break;
+      tc_fence_after_sync();
+      const bool diag = b == i;
+      float mx = -INFINITY;
+#pragma unroll
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem_s + lane_off + c0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int q = 0; q < 32; ++q) {
+          float v = __uint_as_float(r[q]);
+          if (diag && c0 + q > row) v = -INFINITY;
+          mx = fmaxf(mx, v);
+        }
+      }
+      mx *= p.scale_log2;
+      const bool raise = mx > m_used + kRescaleSlack;     // always true for the first block (m_used = -inf)
+      if (__any_sync(0xffffffffu, raise)) {
+        const float m_new = raise ? mx : m_used;
+        const float corr = fast_exp2(m_used - m_new);     // 0 for the first block
+        l_sum *= corr;
+        m_used = m_new;
+        if (j > 0) {
+          if (!(ok = mbar_wait(smem_u32(&bar_pv), (j - 1) & 1, status, kWaitOReady))) break;
+          tc_fence_after_sync();
+#pragma unroll
+          for (int c0 = 0; c0 < 128; c0 += 32) {
+            uint32_t r[32];
+            tmem_ld32(tmem_o + lane_off + c0, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int q = 0; q < 32; ++q) r[q] = __float_as_uint(__uint_as_float(r[q]) * corr);
+            tmem_st32(tmem_o + lane_off + c0, r);
+          }
+        }
+      }
+      const float neg_m = -m_used;
+#pragma unroll
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem_s + lane_off + c0, r);
+        tmem_wait_ld();
+        uint32_t pk[16];
+#pragma unroll
+        for (int q = 0; q < 32; q += 2) {
+          float p0 = fast_exp2(fmaf(__uint_as_float(r[q]), p.scale_log2, neg_m));
+          float p1 = fast_exp2(fmaf(__uint_as_float(r[q + 1]), p.scale_log2, neg_m));
+          if (diag) {
+            if (c0 + q > row) p0 = 0.f;
+            if (c0 + q + 1 > row) p1 = 0.f;
+          }
+          l_sum += p0 + p1;
+          pk[q >> 1] = pack_bf16(p0, p1);
+        }
+        tmem_st16(tmem_s + lane_off + (c0 >> 1), pk);
+      }
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(smem_u32(&bar_p));
+    }
+    // epilogue: O / l -> bf16 -> global
+    __nv_bfloat16* orow = p.O + l * p.osb + (static_cast<int64_t>(i) * B + row) * p.ost + h * p.osh;
+    float* lse_dst = p.lse ? p.lse + (static_cast<int64_t>(l) * p.Hq + h) * p.N + i * B + row : nullptr;
+    if (!any_block) {
+#pragma unroll
+      for (int c = 0; c < 16; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
+      if (lse_dst) *lse_dst = -INFINITY;
+    } else if (ok && mbar_wait(smem_u32(&bar_pv), (j - 1) & 1, status, kWaitOReady)) {
+      tc_fence_after_sync();
+      const float inv = 1.0f / l_sum;
+#pragma unroll
+      for (int c0 = 0; c0 < 128; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem_o + lane_off + c0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int q = 0; q < 32; q += 8) {
+          uint4 v;
+          v.x = pack_bf16(__uint_as_float(r[q]) * inv, __uint_as_float(r[q + 1]) * inv);
+          v.y = pack_bf16(__uint_as_float(r[q + 2]) * inv, __uint_as_float(r[q + 3]) * inv);
+          v.z = pack_bf16(__uint_as_float(r[q + 4]) * inv, __uint_as_float(r[q + 5]) * inv);
+          v.w = pack_bf16(__uint_as_float(r[q + 6]) * inv, __uint_as_float(r[q + 7]) * inv);
+          *reinterpret_cast<uint4*>(orow + c0 + q) = v;
+        }
+      }
+      if (lse_dst) *lse_dst = (m_used + fast_log2(l_sum)) * 0.6931471805599453f;
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  if (warp == 5) tmem_dealloc(s_tmem, 256);
+}
+
+static rbs_status launch_prefill_tc(const PrefillParams& p, const rbs_tensor& Q, const rbs_tensor& K,
+                                    const rbs_tensor& V, int Hkv, cudaStream_t s) {
+  CUtensorMap tmQ, tmK, tmV;
+  rbs_status st;
+  if ((st = make_tmap_lthd(&tmQ, Q.ptr, p.L, p.N, p.Hq, kHeadDim, Q.stride_batch, Q.stride_token, Q.stride_head, 64, 128, true)) != RBS_OK) return st;
+  if ((st = make_tmap_lthd(&tmK, K.ptr, p.L, p.N, Hkv, kHeadDim, K.stride_batch, K.stride_token, K.stride_head, 64, 128, true)) != RBS_OK) return st;
+  if ((st = make_tmap_lthd(&tmV, V.ptr, p.L, p.N, Hkv, kHeadDim, V.stride_batch, V.stride_token, V.stride_head, 64, 128, true)) != RBS_OK) return st;
+  unsigned int* status = device_status_ptr();
+  if (status == nullptr) return RBS_ERR_CUDA;
+  const size_t smem = 3 * 2 * 128 * 128;
+  RBS_CUDA_OK(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.M;
+  if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
+  prefill_tc_kernel<<<static_cast<unsigned>(n_cta), kPfThreads, smem, s>>>(tmQ, tmK, tmV, p, status);
+  RBS_CUDA_OK(cudaGetLastError());
+  return RBS_OK;
+}
+
 template <int B>
 static rbs_status launch_prefill(const PrefillParams& p, cudaStream_t s) {
   const size_t smem = static_cast<size_t>(5) * B * 256;
@@ -221,6 +443,9 @@ static rbs_status launch_prefill(const PrefillParams& p, cudaStream_t s) {
 }
 
 }  // namespace rbs
+
+static int g_prefill_variant = 1;  // 0: mma.sync, 1: tcgen05 (B = 128)
+extern "C" __attribute__((visibility("default"))) void rbs_dev_set_prefill_variant(int v) { g_prefill_variant = v; }
 
 extern "C" rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, rbs_tensor K, rbs_tensor V,
                                          const uint32_t* mask, rbs_tensor O, float* lse, float softmax_scale,
@@ -244,5 +469,6 @@ extern "C" rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, r
   const float scale = softmax_scale == 0.f ? 1.0f / sqrtf(static_cast<float>(x.d)) : softmax_scale;
   p.scale_log2 = scale * kLog2e;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (x.B == 128 && g_prefill_variant == 1) return launch_prefill_tc(p, Q, K, V, x.Hkv, s);
   return (x.B == 128) ? launch_prefill<128>(p, s) : launch_prefill<64>(p, s);
 }
