@@ -167,6 +167,28 @@ def run_reference(args):
 
 
 # ------------------------------------------------------------------------------------------------
+# rank plumbing (replicas only: no data-path collective)
+# ------------------------------------------------------------------------------------------------
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The timed region's duration is the slowest rank's."""
+    if world <= 1:
+        return ms
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def ms_per_layer(ms_per_step: float, world: int, layers_per_rank: int) -> float:
+    """Whole-job figure for a time-like metric: every rank processes `layers_per_rank` layers per step."""
+    return ms_per_step / (world * layers_per_rank)
+
+
+def replica_seed(base_seed: int, rank: int) -> int:
+    return base_seed + rank
+
+
+# ------------------------------------------------------------------------------------------------
 # CUDA leg
 # ------------------------------------------------------------------------------------------------
 def run_ours(args):
@@ -186,7 +208,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
     peaks = load_peaks()
     cfg = workload(args.workload)
-    cfg.seed += rank                       # independent replica per rank
+    cfg.seed = replica_seed(cfg.seed, rank)   # independent replica per rank
     Q, K, V = make_inputs(cfg)
     Qh, Kh, Vh = Q.pin_memory(), K.pin_memory(), V.pin_memory()
     Oh = torch.empty_like(Qh).pin_memory()
@@ -235,10 +257,7 @@ def run_ours(args):
     t_wall1 = time.time()
     total_ms = e0.elapsed_time(e1)
     clocks = sampler.stop(t_wall0, t_wall1) if sampler else None
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, dev)
     ms_per_step = total_ms / args.steps
     t_stats = statistics.mean(ev[0].elapsed_time(ev[1]) for ev in events)
     t_select = statistics.mean(ev[1].elapsed_time(ev[2]) for ev in events)
@@ -258,10 +277,7 @@ def run_ours(args):
     e1.record(stream)
     barrier()
     e2e_ms = e0.elapsed_time(e1) / n_e2e
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = max_over_ranks(e2e_ms, world, dev)
     h2d = Qh.numel() * 2 + Kh.numel() * 2 + Vh.numel() * 2
     d2h = Oh.numel() * 2
 
@@ -314,7 +330,7 @@ def run_ours(args):
         cfg0 = workload(args.workload)
         cpu_ms, cpu_sample, cpu_parts = oracle_sample_ms_per_layer(cfg0, Q, K, V, n_heads=1, n_att_rows=24)
 
-    value = ms_per_step / (world * L)
+    value = ms_per_layer(ms_per_step, world, L)
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": False, "scaling": "weak",
@@ -326,7 +342,7 @@ def run_ours(args):
                      "flops_per_launch_useful": useful, "flops_per_launch_executed": executed},
         "cpu_baseline": ({"value": cpu_ms, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                           "sample": cpu_sample, "parts": cpu_parts} if cpu_ms is not None else None),
-        "e2e": {"value": e2e_ms / (world * L), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
+        "e2e": {"value": ms_per_layer(e2e_ms, world, L), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
         "gpu_launches": 6 * args.steps,
         "clocks": clocks,
         "detail": {
