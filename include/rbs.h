@@ -127,6 +127,37 @@ RBS_API rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, rbs_
                               void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * rbs_select for callers that have no device memory to hand over and must not allocate any.
+ * (The paper has no counterpart: this is a packaging variant of rbs_select, same arithmetic, same outputs.)
+ *
+ * Who needs it: code that runs after the application has claimed the whole GPU for its own pools (a
+ * serving engine that sized its KV cache to the last free byte, so a cudaMalloc would fail or evict),
+ * code on a latency-critical path where the implicit device-wide synchronisation of cudaMalloc/cudaFree
+ * is not acceptable, and plug-ins that are called from inside someone else's memory-managed region and
+ * are simply not given an allocator.  Such callers still pass Q, the statistics and the output buffers;
+ * only the scratch space differs.
+ *
+ * The scratch lives in a fixed array of RBS_SELECT_STATIC_SCRATCH_BYTES inside the library's device
+ * image: every GPU on which the library is loaded holds that much memory until the process exits.
+ * Shapes whose rbs_workspace_bytes(RBS_OP_SELECT) exceed it are rejected with RBS_ERR_WORKSPACE and
+ * nothing is launched (the limit covers about 8,100 centroid rows = batch * n_kv_heads * M rounded up to 128,
+ * e.g. one 128K-token layer with 4 KV heads at block 128 needs about half of it).
+ * The call itself performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ * The first call on each device looks up the array's device address (and, like any first use of a CUDA
+ * module, lets the driver load the kernels); make that first call outside stream capture.
+ * All calls on one device share the one array: it keeps whatever the previous call left there, the
+ * parts that must start at zero are cleared by every call, and two calls whose kernels may overlap on
+ * the GPU (different streams without an ordering between them) race on it -- order them.
+ * Calls to rbs_select with a caller-owned workspace are unaffected.
+ * Arguments, outputs and error codes are those of rbs_select.
+ */
+#define RBS_SELECT_STATIC_SCRATCH_BYTES (4u << 20)
+RBS_API rbs_status rbs_select_static(const rbs_shape* shape, rbs_tensor Q, rbs_stats stats, float alpha_base,
+                                     float alpha_rescue, int n_sink, int n_local, int n_recent, uint32_t* mask,
+                                     float* density, uint32_t* dbg_base_mask, uint32_t* dbg_rescue_mask,
+                                     void* stream);
+
+/*
  * Kernels that wait on hardware barriers (TMA arrival, tensor-core completion) give every wait an
  * iteration limit.  A wait that runs out records a non-zero code in a device-side status word, lets the
  * kernel drain and return, and leaves the CUDA context usable; outputs of that launch are then

@@ -56,6 +56,8 @@ def load_library() -> ctypes.CDLL:
     lib.rbs_block_stats.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, vp]
     lib.rbs_select.restype = i
     lib.rbs_select.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, f, f, i, i, i, vp, vp, vp, vp, vp, sz, vp]
+    lib.rbs_select_static.restype = i
+    lib.rbs_select_static.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, f, f, i, i, i, vp, vp, vp, vp, vp]
     lib.rbs_sparse_prefill.restype = i
     lib.rbs_sparse_prefill.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsTensor, RbsTensor, vp, RbsTensor,
                                        vp, f, vp, sz, vp]
@@ -153,6 +155,26 @@ def rbs_select(Q: torch.Tensor, stats: BlockStats, block: int, alpha_base: float
                           _ptr(workspace), workspace.numel(), _stream()), "rbs_select")
     if debug:
         return mask, density, dbg_b, dbg_r
+    return mask, density
+
+
+SELECT_STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def rbs_select_static(Q: torch.Tensor, stats: BlockStats, block: int, alpha_base: float = 0.22,
+                      alpha_rescue: float = 0.18, n_sink: int = 1, n_local: int = 1, n_recent: int = 1, *,
+                      mask: torch.Tensor, density: torch.Tensor, dbg_base: torch.Tensor | None = None,
+                      dbg_rescue: torch.Tensor | None = None):
+    """rbs_select for callers that may not allocate: the scratch is a fixed array inside the library, and
+    this wrapper allocates nothing either, so `mask` [L,Hq,M,W] int32 and `density` [L,Hq] fp32 must be
+    passed in.  Raises RbsError(RBS_ERR_WORKSPACE) when the shape needs more than
+    SELECT_STATIC_SCRATCH_BYTES of scratch.  Calls on one device share the array: do not let two overlap."""
+    lib = load_library()
+    L, N, Hq, d = Q.shape
+    shape = RbsShape(L, N, Hq, stats.centroid.shape[1], d, block)
+    _check(lib.rbs_select_static(ctypes.byref(shape), _tensor(Q), stats.c_struct(), alpha_base, alpha_rescue,
+                                 n_sink, n_local, n_recent, _ptr(mask), _ptr(density), _ptr(dbg_base),
+                                 _ptr(dbg_rescue), _stream()), "rbs_select_static")
     return mask, density
 
 

@@ -589,3 +589,41 @@ extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats
   RBS_CUDA_OK(cudaGetLastError());
   return RBS_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// rbs_select_static: the same selection for callers that cannot supply or allocate scratch memory.
+// The scratch is this fixed device array.  Its name is only a host-side handle here: the kernels need the
+// device address, which is looked up once per device (with that device current) and then reused.
+// ---------------------------------------------------------------------------------------------
+static __device__ __align__(256) unsigned char g_select_static_scratch[RBS_SELECT_STATIC_SCRATCH_BYTES];
+
+#include <mutex>
+
+extern "C" rbs_status rbs_select_static(const rbs_shape* shape, rbs_tensor Q, rbs_stats stats, float alpha_base,
+                                        float alpha_rescue, int n_sink, int n_local, int n_recent, uint32_t* mask,
+                                        float* density, uint32_t* dbg_base_mask, uint32_t* dbg_rescue_mask,
+                                        void* stream) {
+  using namespace rbs;
+  constexpr int kMaxDevices = 64;
+  static void* scratch_of_device[kMaxDevices] = {nullptr};
+  static std::mutex lock;
+  rbs_status st = check_shape(shape);
+  if (st != RBS_OK) return st;
+  // sizes beyond the fixed array are refused before anything touches the GPU
+  if (select_workspace(make_dims(*shape)).bytes > RBS_SELECT_STATIC_SCRATCH_BYTES) return RBS_ERR_WORKSPACE;
+  int dev = -1;
+  RBS_CUDA_OK(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return RBS_ERR_UNSUPPORTED;
+  void* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> guard(lock);
+    if (scratch_of_device[dev] == nullptr) {
+      void* p = nullptr;
+      if (cudaGetSymbolAddress(&p, g_select_static_scratch) != cudaSuccess || p == nullptr) return RBS_ERR_CUDA;
+      scratch_of_device[dev] = p;
+    }
+    scratch = scratch_of_device[dev];
+  }
+  return rbs_select(shape, Q, stats, alpha_base, alpha_rescue, n_sink, n_local, n_recent, mask, density,
+                    dbg_base_mask, dbg_rescue_mask, scratch, RBS_SELECT_STATIC_SCRATCH_BYTES, stream);
+}
