@@ -61,6 +61,8 @@ def load_library() -> ctypes.CDLL:
     lib.rbs_sparse_prefill.restype = i
     lib.rbs_sparse_prefill.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsTensor, RbsTensor, vp, RbsTensor,
                                        vp, f, vp, sz, vp]
+    lib.rbs_device_status.restype = i
+    lib.rbs_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint), i]
     lib.rbs_status_string.restype = ctypes.c_char_p
     lib.rbs_status_string.argtypes = [i]
     lib.rbs_version.restype = ctypes.c_char_p
@@ -117,6 +119,16 @@ def alloc_stats(K: torch.Tensor, block: int) -> BlockStats:
 
 def workspace_bytes(op: int, shape: RbsShape) -> int:
     return int(load_library().rbs_workspace_bytes(op, ctypes.byref(shape)))
+
+
+def rbs_device_status(clear: bool = True) -> int:
+    """Synchronises the current stream and returns the device status word: 0 unless a bounded wait inside a
+    kernel gave up (the outputs of that launch are then undefined).  `clear` resets the word."""
+    code = ctypes.c_uint(0)
+    rc = load_library().rbs_device_status(_stream(), ctypes.byref(code), 1 if clear else 0)
+    if rc not in (0, 5):
+        _check(rc, "rbs_device_status")
+    return int(code.value)
 
 
 def rbs_block_stats(K: torch.Tensor, block: int, stats: BlockStats | None = None) -> BlockStats:

@@ -218,10 +218,11 @@ prefill_mma_kernel(const PrefillParams p) {
 // other's matrix multiplies.  TMEM columns: [0,128) S, with P (bf16 pairs) written over [0,64) once a
 // thread has read its S row; [128,256) O.
 // Warps 0-3: softmax, one query row per thread (TMEM lane = row).  Warp 4: TMA producer.  Warp 5: MMA issuer.
+// Warps 6-7 only exist so that warps 4-7 form a whole warpgroup that can hand its registers to the softmax warps.
 // The running row maximum is only raised when a block exceeds it by more than kRescaleSlack (log2 units);
 // P then stays below 2^kRescaleSlack and O is rescaled rarely.
 // ---------------------------------------------------------------------------------------------
-constexpr int kPfThreads = 192;
+constexpr int kPfThreads = 256;
 constexpr float kRescaleSlack = 8.0f;
 
 __global__ void __launch_bounds__(kPfThreads, 2)
@@ -236,7 +237,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   unsigned char* sQ = smem;
   unsigned char* sK = smem + kTile;
   unsigned char* sV = smem + 2 * kTile;
-  __shared__ __align__(8) uint64_t bar_q, bar_kfull, bar_vfull, bar_s, bar_p, bar_pv;
+  __shared__ __align__(8) uint64_t bar_q, bar_kfull, bar_vfull, bar_s, bar_p, bar_p1, bar_pv;
   __shared__ uint32_t s_tmem;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -252,6 +253,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     mbar_init(smem_u32(&bar_vfull), 1);
     mbar_init(smem_u32(&bar_s), 1);
     mbar_init(smem_u32(&bar_p), 128);
+    mbar_init(smem_u32(&bar_p1), 128);
     mbar_init(smem_u32(&bar_pv), 1);
     mbar_fence_init();
   }
@@ -261,7 +263,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   tc_fence_after_sync();
   const uint32_t tmem_s = s_tmem, tmem_o = s_tmem + 128;
 
-  if (warp == 4) {
+  if (warp >= 4) reg_dealloc<48>();
+  if (warp >= 6) {
+    // idle: registers donated above
+  } else if (warp == 4) {
     // ------------------------------- TMA producer -------------------------------
     if (lane == 0) {
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -298,18 +303,24 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           mma_ss(tmem_s, smem_desc_sw128(qb + off, 16, 1024), smem_desc_sw128(kb + off, 16, 1024), kIdescQK, k16 != 0);
         }
         mma_commit(smem_u32(&bar_s));
-        if (!(ok = mbar_wait(smem_u32(&bar_p), ph, status, kWaitPReady))) break;
         if (!(ok = mbar_wait(smem_u32(&bar_vfull), ph, status, kWaitTmaFull))) break;
+        if (!(ok = mbar_wait(smem_u32(&bar_p), ph, status, kWaitPReady))) break;    // P columns of keys 0..63
         tc_fence_after_sync();
 #pragma unroll
-        for (int k16 = 0; k16 < 8; ++k16)
+        for (int k16 = 0; k16 < 4; ++k16)
           mma_ts(tmem_o, tmem_s + k16 * 8, smem_desc_sw128(vb + k16 * 2048, kPanel, 1024), kIdescPV, (j | k16) != 0);
+        if (!(ok = mbar_wait(smem_u32(&bar_p1), ph, status, kWaitPReady))) break;   // keys 64..127
+        tc_fence_after_sync();
+#pragma unroll
+        for (int k16 = 4; k16 < 8; ++k16)
+          mma_ts(tmem_o, tmem_s + k16 * 8, smem_desc_sw128(vb + k16 * 2048, kPanel, 1024), kIdescPV, 1);
         mma_commit(smem_u32(&bar_pv));
       }
     }
     __syncwarp();
   } else {
     // ------------------------------- softmax: one query row per thread -------------------------------
+    reg_alloc<208>();
     const int row = warp * 32 + lane;
     const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
     float m_used = -INFINITY, l_sum = 0.f;   // m_used in log2 units of the scaled logits
@@ -317,24 +328,36 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const bool any_block = b >= 0;
     bool ok = true;
     int j = 0;
+    const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
     for (; b >= 0; ++j, b = next_block(mrow, b, i)) {
       if (!(ok = mbar_wait(smem_u32(&bar_s), j & 1, status, kWaitMmaDone))) break;
       tc_fence_after_sync();
-      const bool diag = b == i;
-      float mx = -INFINITY;
-#pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(tmem_s + lane_off + c0, r);
+      uint32_t s[128];   // the whole S row of this thread
+      {
+        uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
+        uint32_t(&s1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32]);
+        uint32_t(&s2)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[64]);
+        uint32_t(&s3)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[96]);
+        tmem_ld32(tmem_s + lane_off, s0);
+        tmem_ld32(tmem_s + lane_off + 32, s1);
+        tmem_ld32(tmem_s + lane_off + 64, s2);
+        tmem_ld32(tmem_s + lane_off + 96, s3);
         tmem_wait_ld();
-#pragma unroll
-        for (int q = 0; q < 32; ++q) {
-          float v = __uint_as_float(r[q]);
-          if (diag && c0 + q > row) v = -INFINITY;
-          mx = fmaxf(mx, v);
-        }
       }
-      mx *= p.scale_log2;
+      if (b == i) {   // diagonal block: keys after the query are hidden
+#pragma unroll
+        for (int c = 0; c < 128; ++c)
+          if (c > row) s[c] = 0xff800000u;   // -inf
+      }
+      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 128; c += 8) {
+        mx0 = max3(mx0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+        mx1 = max3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+        mx2 = max3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
+        mx3 = max3(mx3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
+      }
+      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
       const bool raise = mx > m_used + kRescaleSlack;     // always true for the first block (m_used = -inf)
       if (__any_sync(0xffffffffu, raise)) {
         const float m_new = raise ? mx : m_used;
@@ -355,29 +378,34 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           }
         }
       }
-      const float neg_m = -m_used;
+      const uint64_t negm2 = f2_pack(-m_used, -m_used);
+      uint64_t sum_a = 0ull, sum_b = 0ull;   // (0.f, 0.f)
 #pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(tmem_s + lane_off + c0, r);
-        tmem_wait_ld();
-        uint32_t pk[16];
+      for (int half = 0; half < 2; ++half) {
+        uint32_t pk[32];
 #pragma unroll
-        for (int q = 0; q < 32; q += 2) {
-          float p0 = fast_exp2(fmaf(__uint_as_float(r[q]), p.scale_log2, neg_m));
-          float p1 = fast_exp2(fmaf(__uint_as_float(r[q + 1]), p.scale_log2, neg_m));
-          if (diag) {
-            if (c0 + q > row) p0 = 0.f;
-            if (c0 + q + 1 > row) p1 = 0.f;
-          }
-          l_sum += p0 + p1;
+        for (int q = 0; q < 64; q += 4) {
+          const int c = half * 64 + q;
+          const uint64_t x01 = f2_fma(f2_pack(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), scale2, negm2);
+          const uint64_t x23 = f2_fma(f2_pack(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), scale2, negm2);
+          float x0, x1, x2, x3;
+          f2_unpack(x01, x0, x1);
+          f2_unpack(x23, x2, x3);
+          const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
+          sum_a = f2_add(sum_a, f2_pack(p0, p1));
+          sum_b = f2_add(sum_b, f2_pack(p2, p3));
           pk[q >> 1] = pack_bf16(p0, p1);
+          pk[(q >> 1) + 1] = pack_bf16(p2, p3);
         }
-        tmem_st16(tmem_s + lane_off + (c0 >> 1), pk);
+        tmem_st32(tmem_s + lane_off + half * 32, pk);
+        tmem_wait_st();
+        tc_fence_before_sync();
+        mbar_arrive(smem_u32(half == 0 ? &bar_p : &bar_p1));
       }
-      tmem_wait_st();
-      tc_fence_before_sync();
-      mbar_arrive(smem_u32(&bar_p));
+      float a0, a1, a2, a3;
+      f2_unpack(sum_a, a0, a1);
+      f2_unpack(sum_b, a2, a3);
+      l_sum += (a0 + a1) + (a2 + a3);
     }
     // epilogue: O / l -> bf16 -> global
     __nv_bfloat16* orow = p.O + l * p.osb + (static_cast<int64_t>(i) * B + row) * p.ost + h * p.osh;

@@ -24,6 +24,14 @@ OUT_MAX_ABS = 2e-2
 OUT_MEAN_ABS = 2e-3
 
 
+@pytest.fixture(autouse=True)
+def no_wait_gave_up():
+    """Every kernel wait is bounded; a wait that ran out would leave a code in the device status word."""
+    yield
+    from paper_2609_20971_b200 import rbs_device_status
+    assert rbs_device_status(clear=True) == 0
+
+
 def unpack_mask(mask: torch.Tensor, M: int) -> np.ndarray:
     """[L, Hq, M, W] int32 words -> bool [L, Hq, M, M]."""
     words = mask.cpu().numpy().view(np.uint32)
