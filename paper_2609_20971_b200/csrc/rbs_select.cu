@@ -13,7 +13,7 @@
 namespace rbs {
 
 // ---------------------------------------------------------------------------------------------
-// 1. per (l, KV head): sort radii, quantiles, beta, g = r * beta * scale * log2(e)
+// 1. per (l, KV head): sort radii, quantiles, beta, g = r * beta
 // ---------------------------------------------------------------------------------------------
 constexpr int kCoeffThreads = 1024;
 
@@ -61,7 +61,7 @@ rescue_coeff_kernel(const float* __restrict__ radius, int M, int P /* pow2 >= M 
       bt = live ? fminf(fmaxf((rb - r_low) * inv, 0.f), 1.f) : 0.f;
       beta[static_cast<int64_t>(hd) * M + idx] = bt;
     }
-    g[static_cast<int64_t>(hd) * Mpad + idx] = rb * bt * scale_log2;
+    g[static_cast<int64_t>(hd) * Mpad + idx] = rb * bt;
   }
 }
 
@@ -93,11 +93,14 @@ __global__ void split_centroid_kernel(const float* __restrict__ centroid, int M,
 }
 
 // ---------------------------------------------------------------------------------------------
-// 3. scoring + thresholds + union + pack, one CTA per (l, query head, query block)
+// 3. scoring + thresholds + union + pack on the 5th-generation tensor cores, one CTA per
+//    (batch, query head, query block), two CTAs per SM.
+//   D[128 centroids x B tokens] (fp32, tensor memory) = C_hi . Q_i^T + C_lo . Q_i^T, 16 tcgen05.mma per tile.
+//   One TMEM lane = one centroid, so the aggregation over the block's tokens is a per-thread loop over
+//   the accumulator row: no cross-thread reduction at all.
+// Warps 0-3: epilogue (TMEM lane = centroid row), warp 4: TMA producer, warp 5: MMA issuer and TMEM owner.
+// Two TMEM accumulators let the MMAs of tile t+1 run under the epilogue of tile t.
 // ---------------------------------------------------------------------------------------------
-constexpr int kSelThreads = 256;
-constexpr int kSelTileRows = 128;  // centroid rows per tile
-
 struct SelectParams {
   const __nv_bfloat16* Q; int64_t qsb, qst, qsh;
   const __nv_bfloat16* chi; const __nv_bfloat16* clo; const float* g;
@@ -108,187 +111,10 @@ struct SelectParams {
   unsigned int* counts;
 };
 
-template <int B>
-__global__ void __launch_bounds__(kSelThreads)
-select_kernel(const SelectParams p) {
-  constexpr int NT = B / 8;  // n-tiles (tokens) per warp row-slab
-  extern __shared__ __align__(1024) unsigned char smem[];
-  unsigned char* sQ = smem;                                  // B x 256 B
-  unsigned char* sChi = sQ + B * 256;                        // 128 x 256 B
-  unsigned char* sClo = sChi + kSelTileRows * 256;           // 128 x 256 B
-  float* sQn = reinterpret_cast<float*>(sClo + kSelTileRows * 256);  // B
-  float* sRed = sQn + B;                                     // 32
-  float* sLb = sRed + 32;                                    // n_tiles * 128
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-
-  // heavy query blocks (large i) first
-  const int per_i = p.L * p.Hq;
-  const int i = p.M - 1 - static_cast<int>(blockIdx.x / per_i);
-  const int rem = static_cast<int>(blockIdx.x % per_i);
-  const int l = rem / p.Hq, h = rem % p.Hq, hk = h / p.G;
-  const int Hkv = p.Hq / p.G;
-  const int n_tiles = i / kSelTileRows + 1;
-  float* sLr = sLb + n_tiles * kSelTileRows;
-
-  const __nv_bfloat16* qbase = p.Q + l * p.qsb + static_cast<int64_t>(i) * B * p.qst + h * p.qsh;
-  const int64_t crow0 = (static_cast<int64_t>(l) * Hkv + hk) * p.Mpad;
-
-  auto load_ctile = [&](int bt) {
-    for (int c = tid; c < kSelTileRows * 16; c += kSelThreads) {
-      const int row = c >> 4, chunk = c & 15;
-      const int64_t src = (crow0 + bt * kSelTileRows + row) * kHeadDim + chunk * 8;
-      cp_async16(smem_u32(sChi + tile_off(row, chunk)), p.chi + src);
-      cp_async16(smem_u32(sClo + tile_off(row, chunk)), p.clo + src);
-    }
-  };
-
-  for (int c = tid; c < B * 16; c += kSelThreads) {
-    const int row = c >> 4, chunk = c & 15;
-    cp_async16(smem_u32(sQ + tile_off(row, chunk)), qbase + static_cast<int64_t>(row) * p.qst + chunk * 8);
-  }
-  load_ctile(0);
-  cp_async_commit();
-  cp_async_wait<0>();
-  __syncthreads();
-
-  // raw query norms ||q_t||_2
-  if (tid < B) {
-    float s = 0.f;
-#pragma unroll
-    for (int chunk = 0; chunk < 16; ++chunk) {
-      const uint4 v = *reinterpret_cast<const uint4*>(sQ + tile_off(tid, chunk));
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const float a = bf16lo(w[k]), c = bf16hi(w[k]);
-        s = fmaf(a, a, s);
-        s = fmaf(c, c, s);
-      }
-    }
-    sQn[tid] = sqrtf(s);
-  }
-  __syncthreads();
-
-  const int gq = lane >> 2, tq = lane & 3;
-  for (int bt = 0; bt < n_tiles; ++bt) {
-    float acc[NT][4];
-#pragma unroll
-    for (int nt = 0; nt < NT; ++nt) { acc[nt][0] = acc[nt][1] = acc[nt][2] = acc[nt][3] = 0.f; }
-#pragma unroll
-    for (int k16 = 0; k16 < 8; ++k16) {
-      uint32_t ahi[4], alo[4];
-      const uint32_t aoff = tile_off(warp * 16 + (lane & 15), 2 * k16 + (lane >> 4));
-      ldmatrix_x4(ahi[0], ahi[1], ahi[2], ahi[3], smem_u32(sChi + aoff));
-      ldmatrix_x4(alo[0], alo[1], alo[2], alo[3], smem_u32(sClo + aoff));
-#pragma unroll
-      for (int ntp = 0; ntp < NT / 2; ++ntp) {
-        uint32_t b0, b1, b2, b3;
-        const int row = 16 * ntp + (lane & 7) + ((lane >> 4) << 3);
-        ldmatrix_x4(b0, b1, b2, b3, smem_u32(sQ + tile_off(row, 2 * k16 + ((lane >> 3) & 1))));
-        mma_bf16_16816(acc[2 * ntp], ahi, b0, b1);
-        mma_bf16_16816(acc[2 * ntp], alo, b0, b1);
-        mma_bf16_16816(acc[2 * ntp + 1], ahi, b2, b3);
-        mma_bf16_16816(acc[2 * ntp + 1], alo, b2, b3);
-      }
-    }
-    // per centroid row: log2-sum-exp2 over the block's tokens, both branches
-#pragma unroll
-    for (int rr = 0; rr < 2; ++rr) {
-      const int b = bt * kSelTileRows + warp * 16 + gq + rr * 8;
-      const float gb = p.g[crow0 + b];
-      float mb = -INFINITY, mr = -INFINITY;
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        const float2 qn = *reinterpret_cast<const float2*>(sQn + nt * 8 + tq * 2);
-        const float x0 = acc[nt][2 * rr] * p.scale_log2, x1 = acc[nt][2 * rr + 1] * p.scale_log2;
-        acc[nt][2 * rr] = x0; acc[nt][2 * rr + 1] = x1;
-        mb = fmaxf(mb, fmaxf(x0, x1));
-        mr = fmaxf(mr, fmaxf(fmaf(qn.x, gb, x0), fmaf(qn.y, gb, x1)));
-      }
-      mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, 1));
-      mb = fmaxf(mb, __shfl_xor_sync(0xffffffffu, mb, 2));
-      mr = fmaxf(mr, __shfl_xor_sync(0xffffffffu, mr, 1));
-      mr = fmaxf(mr, __shfl_xor_sync(0xffffffffu, mr, 2));
-      float sb = 0.f, sr = 0.f;
-#pragma unroll
-      for (int nt = 0; nt < NT; ++nt) {
-        const float2 qn = *reinterpret_cast<const float2*>(sQn + nt * 8 + tq * 2);
-        const float x0 = acc[nt][2 * rr], x1 = acc[nt][2 * rr + 1];
-        sb += fast_exp2(x0 - mb) + fast_exp2(x1 - mb);
-        sr += fast_exp2(fmaf(qn.x, gb, x0) - mr) + fast_exp2(fmaf(qn.y, gb, x1) - mr);
-      }
-      sb += __shfl_xor_sync(0xffffffffu, sb, 1);
-      sb += __shfl_xor_sync(0xffffffffu, sb, 2);
-      sr += __shfl_xor_sync(0xffffffffu, sr, 1);
-      sr += __shfl_xor_sync(0xffffffffu, sr, 2);
-      if (tq == 0) {
-        const bool causal = b <= i;
-        sLb[b] = causal ? mb + fast_log2(sb) : -INFINITY;
-        sLr[b] = causal ? mr + fast_log2(sr) : -INFINITY;
-      }
-    }
-    __syncthreads();  // every warp is done with this centroid tile
-    if (bt + 1 < n_tiles) {
-      load_ctile(bt + 1);
-      cp_async_commit();
-      cp_async_wait<0>();
-      __syncthreads();
-    }
-  }
-
-  // row maxima over the causal candidates
-  float mxb = -INFINITY, mxr = -INFINITY;
-  for (int b = tid; b <= i; b += kSelThreads) { mxb = fmaxf(mxb, sLb[b]); mxr = fmaxf(mxr, sLr[b]); }
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    mxb = fmaxf(mxb, __shfl_xor_sync(0xffffffffu, mxb, o));
-    mxr = fmaxf(mxr, __shfl_xor_sync(0xffffffffu, mxr, o));
-  }
-  if (lane == 0) { sRed[warp] = mxb; sRed[8 + warp] = mxr; }
-  __syncthreads();
-  mxb = sRed[0]; mxr = sRed[8];
-#pragma unroll
-  for (int w = 1; w < kSelThreads / 32; ++w) { mxb = fmaxf(mxb, sRed[w]); mxr = fmaxf(mxr, sRed[8 + w]); }
-  const float thr_b = mxb + p.t_base, thr_r = mxr + p.t_rescue;
-
-  const int64_t mrow = ((static_cast<int64_t>(l) * p.Hq + h) * p.M + i) * p.W;
-  const bool all_forced = i >= p.M - p.n_recent;
-  unsigned int cnt = 0;
-  for (int w = warp; w < p.W; w += kSelThreads / 32) {
-    const int b = w * 32 + lane;
-    const bool valid = b <= i;
-    bool kb = false, kr = false, kf = false;
-    if (valid) {
-      kb = sLb[b] >= thr_b;
-      kr = sLr[b] >= thr_r;
-      kf = all_forced || b < p.n_sink || b > i - p.n_local;
-    }
-    const uint32_t wb = __ballot_sync(0xffffffffu, kb), wr = __ballot_sync(0xffffffffu, kr);
-    const uint32_t wf = __ballot_sync(0xffffffffu, kf);
-    if (lane == 0) {
-      const uint32_t word = wb | wr | wf;
-      p.mask[mrow + w] = word;
-      if (p.dbg_base) p.dbg_base[mrow + w] = wb;
-      if (p.dbg_rescue) p.dbg_rescue[mrow + w] = wr;
-      cnt += __popc(word);
-    }
-  }
-  if (lane == 0 && cnt) atomicAdd(p.counts + l * p.Hq + h, cnt);
-}
-
-// ---------------------------------------------------------------------------------------------
-// 3b. the same scoring on the 5th-generation tensor cores.
-//   D[128 centroids x B tokens] (fp32, tensor memory) = C_hi . Q_i^T + C_lo . Q_i^T, 16 tcgen05.mma per tile.
-//   One TMEM lane = one centroid, so the aggregation over the block's tokens is a per-thread loop over
-//   the accumulator row: no cross-thread reduction at all.
-// Warp roles: warps 0-3 and 4-7 = two epilogue groups (tile parity), warp 8 = TMA producer,
-// warp 9 = MMA issuer and TMEM owner.
-// ---------------------------------------------------------------------------------------------
-constexpr int kTcThreads = 320;
-constexpr int kTcStages = 2;
+constexpr int kTcThreads = 192;
 
 template <int B>
-__global__ void __launch_bounds__(kTcThreads, 1)
+__global__ void __launch_bounds__(kTcThreads, 2)
 select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmChi,
                  const __grid_constant__ CUtensorMap tmClo, const SelectParams p, unsigned int* status) {
   constexpr uint32_t kPanelC = 128 * 128;          // one 64-column panel of a 128-row centroid tile
@@ -296,12 +122,12 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   constexpr uint32_t kPanelQ = B * 128;
   constexpr uint32_t kIdesc = idesc_bf16_f32(128, B, false);
   extern __shared__ __align__(1024) unsigned char smem[];
-  unsigned char* sC = smem;                                        // kTcStages x 64 KB
-  unsigned char* sQ = sC + kTcStages * kStage;                     // 2 panels
+  unsigned char* sC = smem;                                        // 64 KB
+  unsigned char* sQ = sC + kStage;                                 // 2 panels
   float* sQn = reinterpret_cast<float*>(sQ + 2 * kPanelQ);         // B
   float* sRed = sQn + B;                                           // 32
   float* sLb = sRed + 32;
-  __shared__ __align__(8) uint64_t bar_q, bar_cfull[kTcStages], bar_cempty[kTcStages], bar_tfull[2], bar_tempty[2];
+  __shared__ __align__(8) uint64_t bar_q, bar_cfull, bar_cempty, bar_tfull[2], bar_tempty[2];
   __shared__ uint32_t s_tmem;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -316,28 +142,27 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
   if (tid == 0) {
     mbar_init(smem_u32(&bar_q), 1);
-    for (int s = 0; s < kTcStages; ++s) { mbar_init(smem_u32(&bar_cfull[s]), 1); mbar_init(smem_u32(&bar_cempty[s]), 1); }
+    mbar_init(smem_u32(&bar_cfull), 1);
+    mbar_init(smem_u32(&bar_cempty), 1);
     for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bar_tfull[s]), 1); mbar_init(smem_u32(&bar_tempty[s]), 4); }
     mbar_fence_init();
   }
-  if (warp == 9) tmem_alloc(smem_u32(&s_tmem), 2 * B);
+  if (warp == 5) tmem_alloc(smem_u32(&s_tmem), 2 * B);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = s_tmem;
 
-  if (warp == 8) {
+  if (warp == 4) {
     // ------------------------------- TMA producer -------------------------------
     if (lane == 0) {
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmChi); tma_prefetch_desc(&tmClo);
       mbar_arrive_expect_tx(smem_u32(&bar_q), 2 * kPanelQ);
       tma_load_4d(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, i * B, l);
       tma_load_4d(smem_u32(sQ + kPanelQ), &tmQ, smem_u32(&bar_q), 64, h, i * B, l);
+      const uint32_t full = smem_u32(&bar_cfull), dst = smem_u32(sC);
       for (int bt = 0; bt < n_tiles; ++bt) {
-        const int s = bt % kTcStages, use = bt / kTcStages;
-        if (use > 0 && !mbar_wait(smem_u32(&bar_cempty[s]), (use - 1) & 1, status, kWaitStageFree)) break;
-        const uint32_t full = smem_u32(&bar_cfull[s]);
-        const uint32_t dst = smem_u32(sC + s * kStage);
+        if (bt > 0 && !mbar_wait(smem_u32(&bar_cempty), (bt - 1) & 1, status, kWaitStageFree)) break;
         mbar_arrive_expect_tx(full, kStage);
         tma_load_2d(dst, &tmChi, full, 0, crow0 + bt * 128);
         tma_load_2d(dst + kPanelC, &tmChi, full, 64, crow0 + bt * 128);
@@ -345,19 +170,18 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         tma_load_2d(dst + 3 * kPanelC, &tmClo, full, 64, crow0 + bt * 128);
       }
     }
-  } else if (warp == 9) {
+  } else if (warp == 5) {
     // ------------------------------- MMA issuer -------------------------------
     if (lane == 0) {
       bool ok = mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
+      const uint32_t cbase = smem_u32(sC), qbase = smem_u32(sQ);
       for (int bt = 0; ok && bt < n_tiles; ++bt) {
-        const int s = bt % kTcStages, buf = bt & 1;
-        ok = mbar_wait(smem_u32(&bar_cfull[s]), (bt / kTcStages) & 1, status, kWaitTmaFull);
+        const int buf = bt & 1;
+        ok = mbar_wait(smem_u32(&bar_cfull), bt & 1, status, kWaitTmaFull);
         if (ok && bt >= 2) ok = mbar_wait(smem_u32(&bar_tempty[buf]), ((bt >> 1) - 1) & 1, status, kWaitTmemFree);
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + buf * B;
-        const uint32_t cbase = smem_u32(sC + s * kStage);
-        const uint32_t qbase = smem_u32(sQ);
 #pragma unroll
         for (int half = 0; half < 2; ++half) {
 #pragma unroll
@@ -367,18 +191,16 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
             mma_ss(d_tmem, adesc, bdesc, kIdesc, (half | k16) != 0);
           }
         }
-        mma_commit(smem_u32(&bar_cempty[s]));
+        mma_commit(smem_u32(&bar_cempty));
         mma_commit(smem_u32(&bar_tfull[buf]));
       }
     }
     __syncwarp();
   } else {
-    // ------------------------------- epilogue groups -------------------------------
-    const int grp = warp >> 2;                       // tile parity handled by this group
-    const int row = (warp & 3) * 32 + lane;          // TMEM lane = centroid row inside the tile
+    // ------------------------------- epilogue: one centroid row per thread -------------------------------
+    const int row = warp * 32 + lane;
     bool ok = mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
-    // raw query norms (both groups compute the half they own; B <= 128 tokens, 256 epilogue threads)
-    if (ok && tid < B) {
+    if (ok && tid < B) {   // raw query norms ||q_t||_2
       float s2 = 0.f;
 #pragma unroll
       for (int c = 0; c < 16; ++c) {
@@ -393,15 +215,19 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
       sQn[tid] = sqrtf(s2);
     }
-    asm volatile("bar.sync 1, 256;" ::: "memory");   // the eight epilogue warps
-    for (int bt = grp; ok && bt < n_tiles; bt += 2) {
-      ok = mbar_wait(smem_u32(&bar_tfull[grp]), (bt >> 1) & 1, status, kWaitMmaDone);
+    asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps
+    const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
+    for (int bt = 0; ok && bt < n_tiles; ++bt) {
+      const int buf = bt & 1;
+      ok = mbar_wait(smem_u32(&bar_tfull[buf]), (bt >> 1) & 1, status, kWaitMmaDone);
       if (!ok) break;
       tc_fence_after_sync();
       const int b = bt * 128 + row;
-      const float gb = p.g[crow0 + b];
-      const uint32_t taddr = tmem_base + grp * B + (static_cast<uint32_t>((warp & 3) * 32) << 16);
-      float mb = -INFINITY, mr = -INFINITY;
+      const float gb = p.g[crow0 + b];            // r_b beta_b, unscaled
+      const uint64_t gb2 = f2_pack(gb, gb);
+      const uint32_t taddr = tmem_base + buf * B + (static_cast<uint32_t>(warp * 32) << 16);
+      // pass 1: maxima of the raw logits x and of y = x + ||q|| r beta
+      float mb0 = -INFINITY, mb1 = -INFINITY, mr0 = -INFINITY, mr1 = -INFINITY;
 #pragma unroll
       for (int c0 = 0; c0 < B; c0 += 32) {
         uint32_t r[32];
@@ -410,14 +236,18 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
         for (int j = 0; j < 32; j += 4) {
           const float4 qn = *reinterpret_cast<const float4*>(sQn + c0 + j);
-          const float x0 = __uint_as_float(r[j]) * p.scale_log2, x1 = __uint_as_float(r[j + 1]) * p.scale_log2;
-          const float x2 = __uint_as_float(r[j + 2]) * p.scale_log2, x3 = __uint_as_float(r[j + 3]) * p.scale_log2;
-          mb = fmaxf(mb, fmaxf(fmaxf(x0, x1), fmaxf(x2, x3)));
-          mr = fmaxf(mr, fmaxf(fmaxf(fmaf(qn.x, gb, x0), fmaf(qn.y, gb, x1)), fmaxf(fmaf(qn.z, gb, x2), fmaf(qn.w, gb, x3))));
+          float y0, y1, y2, y3;
+          f2_unpack(f2_fma(f2_pack(qn.x, qn.y), gb2, f2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1]))), y0, y1);
+          f2_unpack(f2_fma(f2_pack(qn.z, qn.w), gb2, f2_pack(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]))), y2, y3);
+          mb0 = max3(mb0, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+          mb1 = max3(mb1, __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+          mr0 = max3(mr0, y0, y1);
+          mr1 = max3(mr1, y2, y3);
         }
       }
-      float sb = 0.f, sr = 0.f;
-      const float nmb = -mb, nmr = -mr;
+      const float mb = fmaxf(mb0, mb1) * p.scale_log2, mr = fmaxf(mr0, mr1) * p.scale_log2;   // log2 units
+      const uint64_t nmb2 = f2_pack(-mb, -mb), nmr2 = f2_pack(-mr, -mr);
+      uint64_t sb2 = 0ull, sr2 = 0ull, sb2b = 0ull, sr2b = 0ull;
 #pragma unroll
       for (int c0 = 0; c0 < B; c0 += 32) {
         uint32_t r[32];
@@ -426,29 +256,38 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (c0 + 32 >= B) {   // accumulator fully read: hand the TMEM buffer back to the MMA warp
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bar_tempty[grp]));
+          if (lane == 0) mbar_arrive(smem_u32(&bar_tempty[buf]));
         }
 #pragma unroll
         for (int j = 0; j < 32; j += 4) {
           const float4 qn = *reinterpret_cast<const float4*>(sQn + c0 + j);
-          const float x0 = __uint_as_float(r[j]) * p.scale_log2, x1 = __uint_as_float(r[j + 1]) * p.scale_log2;
-          const float x2 = __uint_as_float(r[j + 2]) * p.scale_log2, x3 = __uint_as_float(r[j + 3]) * p.scale_log2;
-          sb += fast_exp2(x0 + nmb) + fast_exp2(x1 + nmb) + fast_exp2(x2 + nmb) + fast_exp2(x3 + nmb);
-          sr += fast_exp2(fmaf(qn.x, gb, x0) + nmr) + fast_exp2(fmaf(qn.y, gb, x1) + nmr) +
-                fast_exp2(fmaf(qn.z, gb, x2) + nmr) + fast_exp2(fmaf(qn.w, gb, x3) + nmr);
+          const uint64_t x01 = f2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+          const uint64_t x23 = f2_pack(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+          float e0, e1, e2, e3, f0, f1, f2, f3;
+          f2_unpack(f2_fma(x01, scale2, nmb2), e0, e1);
+          f2_unpack(f2_fma(x23, scale2, nmb2), e2, e3);
+          f2_unpack(f2_fma(f2_fma(f2_pack(qn.x, qn.y), gb2, x01), scale2, nmr2), f0, f1);
+          f2_unpack(f2_fma(f2_fma(f2_pack(qn.z, qn.w), gb2, x23), scale2, nmr2), f2, f3);
+          sb2 = f2_add(sb2, f2_pack(fast_exp2(e0), fast_exp2(e1)));
+          sb2b = f2_add(sb2b, f2_pack(fast_exp2(e2), fast_exp2(e3)));
+          sr2 = f2_add(sr2, f2_pack(fast_exp2(f0), fast_exp2(f1)));
+          sr2b = f2_add(sr2b, f2_pack(fast_exp2(f2), fast_exp2(f3)));
         }
       }
+      float a0, a1, a2, a3;
+      f2_unpack(f2_add(sb2, sb2b), a0, a1);
+      f2_unpack(f2_add(sr2, sr2b), a2, a3);
       const bool causal = b <= i;
-      sLb[b] = causal ? mb + fast_log2(sb) : -INFINITY;
-      sLr[b] = causal ? mr + fast_log2(sr) : -INFINITY;
+      sLb[b] = causal ? mb + fast_log2(a0 + a1) : -INFINITY;
+      sLr[b] = causal ? mr + fast_log2(a2 + a3) : -INFINITY;
     }
   }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  if (warp == 9) tmem_dealloc(tmem_base, 2 * B);
+  if (warp == 5) tmem_dealloc(tmem_base, 2 * B);
 
-  // row maxima over the causal candidates, thresholds, forced blocks, union, pack (all ten warps)
+  // row maxima over the causal candidates, thresholds, forced blocks, union, pack (all six warps)
   float mxb = -INFINITY, mxr = -INFINITY;
   for (int b = tid; b <= i; b += kTcThreads) { mxb = fmaxf(mxb, sLb[b]); mxr = fmaxf(mxr, sLr[b]); }
 #pragma unroll
@@ -496,19 +335,6 @@ __global__ void density_kernel(const unsigned int* __restrict__ counts, int n, i
 }
 
 template <int B>
-static rbs_status launch_select(const SelectParams& p, cudaStream_t s) {
-  const int n_tiles_max = (p.M + kSelTileRows - 1) / kSelTileRows;
-  const size_t smem = static_cast<size_t>(B) * 256 + 2 * kSelTileRows * 256 + (B + 32) * sizeof(float) +
-                      2 * static_cast<size_t>(n_tiles_max) * kSelTileRows * sizeof(float);
-  RBS_CUDA_OK(cudaFuncSetAttribute(select_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-  const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.M;
-  if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
-  select_kernel<B><<<static_cast<unsigned>(n_cta), kSelThreads, smem, s>>>(p);
-  RBS_CUDA_OK(cudaGetLastError());
-  return RBS_OK;
-}
-
-template <int B>
 static rbs_status launch_select_tc(const SelectParams& p, const rbs_tensor& Q, int N, cudaStream_t s) {
   CUtensorMap tmQ, tmChi, tmClo;
   rbs_status st = make_tmap_lthd(&tmQ, Q.ptr, p.L, N, p.Hq, kHeadDim, Q.stride_batch, Q.stride_token, Q.stride_head, 64, B, true);
@@ -519,7 +345,7 @@ static rbs_status launch_select_tc(const SelectParams& p, const rbs_tensor& Q, i
   unsigned int* status = device_status_ptr();
   if (status == nullptr) return RBS_ERR_CUDA;
   const int n_tiles_max = (p.M + 127) / 128;
-  const size_t smem = static_cast<size_t>(kTcStages) * 4 * 128 * 128 + 2 * static_cast<size_t>(B) * 128 +
+  const size_t smem = static_cast<size_t>(4) * 128 * 128 + 2 * static_cast<size_t>(B) * 128 +
                       (B + 32) * sizeof(float) + 2 * static_cast<size_t>(n_tiles_max) * 128 * sizeof(float);
   auto kern = select_tc_kernel<B>;
   RBS_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
@@ -531,9 +357,6 @@ static rbs_status launch_select_tc(const SelectParams& p, const rbs_tensor& Q, i
 }
 
 }  // namespace rbs
-
-static int g_select_variant = 1;  // 0: mma.sync, 1: tcgen05
-extern "C" __attribute__((visibility("default"))) void rbs_dev_set_select_variant(int v) { g_select_variant = v; }
 
 extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats stats, float alpha_base,
                                  float alpha_rescue, int n_sink, int n_local, int n_recent, uint32_t* mask,
@@ -579,10 +402,7 @@ extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats
   p.scale_log2 = scale_log2; p.t_base = log2f(alpha_base); p.t_rescue = log2f(alpha_rescue);
   p.n_sink = n_sink; p.n_local = n_local; p.n_recent = n_recent;
   p.mask = mask; p.dbg_base = dbg_base_mask; p.dbg_rescue = dbg_rescue_mask; p.counts = counts;
-  if (g_select_variant == 1)
-    st = (x.B == 128) ? launch_select_tc<128>(p, Q, x.N, s) : launch_select_tc<64>(p, Q, x.N, s);
-  else
-    st = (x.B == 128) ? launch_select<128>(p, s) : launch_select<64>(p, s);
+  st = (x.B == 128) ? launch_select_tc<128>(p, Q, x.N, s) : launch_select_tc<64>(p, Q, x.N, s);
   if (st != RBS_OK) return st;
   const int nh = x.L * x.Hq;
   density_kernel<<<(nh + 127) / 128, 128, 0, s>>>(counts, nh, x.M, density);
