@@ -289,32 +289,50 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     }
   } else if (warp == 5) {
     // ------------------------------- MMA issuer -------------------------------
+    // Everything this thread does between two waits sits on the critical path of the tile, so the operand
+    // descriptors are built once (they only differ in the address field) and the next block index is
+    // fetched from the mask while the softmax of the current block runs.
     if (lane == 0) {
       int b = next_block(mrow, -1, i);
       bool ok = b < 0 || mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
-      const uint32_t qb = smem_u32(sQ), kb = smem_u32(sK), vb = smem_u32(sV);
-      for (int j = 0; ok && b >= 0; ++j, b = next_block(mrow, b, i)) {
-        const uint32_t ph = j & 1;
-        if (!(ok = mbar_wait(smem_u32(&bar_kfull), ph, status, kWaitTmaFull))) break;
-        tc_fence_after_sync();
+      const uint64_t dq = smem_desc_sw128(smem_u32(sQ), 16, 1024);
+      const uint64_t dk = smem_desc_sw128(smem_u32(sK), 16, 1024);
+      const uint64_t dv = smem_desc_sw128(smem_u32(sV), kPanel, 1024);
+      auto issue_qk = [&]() {
 #pragma unroll
         for (int k16 = 0; k16 < 8; ++k16) {
-          const uint32_t off = (k16 >> 2) * kPanel + (k16 & 3) * 32;
-          mma_ss(tmem_s, smem_desc_sw128(qb + off, 16, 1024), smem_desc_sw128(kb + off, 16, 1024), kIdescQK, k16 != 0);
+          const uint64_t off = static_cast<uint64_t>(((k16 >> 2) * kPanel + (k16 & 3) * 32) >> 4);
+          mma_ss(tmem_s, dq + off, dk + off, kIdescQK, k16 != 0);
         }
         mma_commit(smem_u32(&bar_s));
+      };
+      if (ok && b >= 0) {
+        if ((ok = mbar_wait(smem_u32(&bar_kfull), 0, status, kWaitTmaFull))) {
+          tc_fence_after_sync();
+          issue_qk();
+        }
+      }
+      for (int j = 0; ok && b >= 0; ++j) {
+        const uint32_t ph = j & 1;
+        const int b_next = next_block(mrow, b, i);     // global-memory latency hidden behind the softmax
         if (!(ok = mbar_wait(smem_u32(&bar_vfull), ph, status, kWaitTmaFull))) break;
         if (!(ok = mbar_wait(smem_u32(&bar_p), ph, status, kWaitPReady))) break;    // P columns of keys 0..63
         tc_fence_after_sync();
 #pragma unroll
         for (int k16 = 0; k16 < 4; ++k16)
-          mma_ts(tmem_o, tmem_s + k16 * 8, smem_desc_sw128(vb + k16 * 2048, kPanel, 1024), kIdescPV, (j | k16) != 0);
+          mma_ts(tmem_o, tmem_s + k16 * 8, dv + static_cast<uint64_t>((k16 * 2048) >> 4), kIdescPV, (j | k16) != 0);
         if (!(ok = mbar_wait(smem_u32(&bar_p1), ph, status, kWaitPReady))) break;   // keys 64..127
         tc_fence_after_sync();
 #pragma unroll
         for (int k16 = 4; k16 < 8; ++k16)
-          mma_ts(tmem_o, tmem_s + k16 * 8, smem_desc_sw128(vb + k16 * 2048, kPanel, 1024), kIdescPV, 1);
+          mma_ts(tmem_o, tmem_s + k16 * 8, dv + static_cast<uint64_t>((k16 * 2048) >> 4), kIdescPV, 1);
         mma_commit(smem_u32(&bar_pv));
+        if (b_next >= 0) {                              // K of the next block arrived while the softmax ran
+          if (!(ok = mbar_wait(smem_u32(&bar_kfull), ph ^ 1, status, kWaitTmaFull))) break;
+          tc_fence_after_sync();
+          issue_qk();
+        }
+        b = b_next;
       }
     }
     __syncwarp();
@@ -349,15 +367,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         for (int c = 0; c < 128; ++c)
           if (c > row) s[c] = 0xff800000u;   // -inf
       }
-      float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+      float mxa[8];
 #pragma unroll
-      for (int c = 0; c < 128; c += 8) {
-        mx0 = max3(mx0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
-        mx1 = max3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
-        mx2 = max3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
-        mx3 = max3(mx3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
+      for (int u = 0; u < 8; ++u) mxa[u] = -INFINITY;
+#pragma unroll
+      for (int c = 0; c < 128; c += 16) {
+#pragma unroll
+        for (int u = 0; u < 8; ++u) mxa[u] = max3(mxa[u], __uint_as_float(s[c + 2 * u]), __uint_as_float(s[c + 2 * u + 1]));
       }
-      const float mx = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)) * p.scale_log2;
+      const float mx = fmaxf(max3(mxa[0], mxa[1], mxa[2]), max3(max3(mxa[3], mxa[4], mxa[5]), mxa[6], mxa[7])) * p.scale_log2;
       const bool raise = mx > m_used + kRescaleSlack;     // always true for the first block (m_used = -inf)
       if (__any_sync(0xffffffffu, raise)) {
         const float m_new = raise ? mx : m_used;
