@@ -224,6 +224,9 @@ prefill_mma_kernel(const PrefillParams p) {
 // ---------------------------------------------------------------------------------------------
 constexpr int kPfThreads = 256;
 constexpr float kRescaleSlack = 8.0f;
+// Of every (kPolyEvery + 1) groups of four logits, one pair is exponentiated by polynomial (0: every group
+// = 50 % of the exps, 1: 25 %, 3: 12.5 %).
+constexpr int kPolyEvery = 1;
 
 __global__ void __launch_bounds__(kPfThreads, 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -409,7 +412,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           float x0, x1, x2, x3;
           f2_unpack(x01, x0, x1);
           f2_unpack(x23, x2, x3);
-          const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
+          const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+          float p2, p3;
+          if (((q >> 2) & kPolyEvery) == kPolyEvery) {   // a share of the exps goes to the FMA pipe
+            exp2_poly_x2(x23, p2, p3);
+          } else {
+            p2 = fast_exp2(x2);
+            p3 = fast_exp2(x3);
+          }
           sum_a = f2_add(sum_a, f2_pack(p0, p1));
           sum_b = f2_add(sum_b, f2_pack(p2, p3));
           pk[q >> 1] = pack_bf16(p0, p1);

@@ -203,4 +203,31 @@ __device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b) {
   return d;
 }
 
+__device__ __forceinline__ uint64_t f2_add_rm(uint64_t a, uint64_t b) {   // round toward -inf
+  uint64_t d;
+  asm("add.rm.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+
+// 2^x for two values on the FMA pipe instead of the special-function unit (which is the scarce unit in
+// the softmax): x = n + f with n = floor(x), 2^f by a degree-3 minimax polynomial on [0, 1) (relative
+// error 7.5e-5), then n is added into the exponent field.  Inputs are clamped to x >= -126; x <= 127.
+__device__ __forceinline__ void exp2_poly_x2(uint64_t x2, float& r0, float& r1) {
+  constexpr float kMagic = 12582912.0f;   // 1.5 * 2^23: its float spacing is 1
+  float x0, x1;
+  f2_unpack(x2, x0, x1);
+  const uint64_t xc = f2_pack(fmaxf(x0, -126.0f), fmaxf(x1, -126.0f));
+  const uint64_t t = f2_add_rm(xc, f2_pack(kMagic, kMagic));                  // low mantissa bits = floor(x)
+  const uint64_t fl = f2_add(t, f2_pack(-kMagic, -kMagic));                   // floor(x), exact
+  const uint64_t f = f2_fma(fl, f2_pack(-1.0f, -1.0f), xc);                   // x - floor(x) in [0, 1)
+  uint64_t pl = f2_fma(f, f2_pack(0.0780242234f, 0.0780242234f), f2_pack(0.2260672301f, 0.2260672301f));
+  pl = f2_fma(pl, f, f2_pack(0.6958336830f, 0.6958336830f));
+  pl = f2_fma(pl, f, f2_pack(0.9999251962f, 0.9999251962f));
+  float p0, p1, t0, t1;
+  f2_unpack(pl, p0, p1);
+  f2_unpack(t, t0, t1);
+  r0 = __int_as_float(__float_as_int(p0) + (__float_as_int(t0) << 23));
+  r1 = __int_as_float(__float_as_int(p1) + (__float_as_int(t1) << 23));
+}
+
 }  // namespace rbs
