@@ -292,10 +292,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     }
   } else if (warp == 5) {
     // ------------------------------- MMA issuer -------------------------------
-    // Everything this thread does between two waits sits on the critical path of the tile, so the operand
-    // descriptors are built once (they only differ in the address field) and the next block index is
-    // fetched from the mask while the softmax of the current block runs.
-    if (lane == 0) {
+    // The whole warp runs this loop in lock step and one elected lane issues each tcgen05 instruction.
+    // Everything between two waits sits on the critical path of the tile, so the operand descriptors are
+    // built once (they only differ in the address field) and the next block index is fetched from the
+    // mask while the softmax of the current block runs.
+    {
       int b = next_block(mrow, -1, i);
       bool ok = b < 0 || mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
       const uint64_t dq = smem_desc_sw128(smem_u32(sQ), 16, 1024);
@@ -305,12 +306,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 #pragma unroll
         for (int k16 = 0; k16 < 8; ++k16) {
           const uint64_t off = static_cast<uint64_t>(((k16 >> 2) * kPanel + (k16 & 3) * 32) >> 4);
-          mma_ss(tmem_s, dq + off, dk + off, kIdescQK, k16 != 0);
+          mma_ss_elect(tmem_s, dq + off, dk + off, kIdescQK, k16 != 0);
         }
-        mma_commit(smem_u32(&bar_s));
+        mma_commit_elect(smem_u32(&bar_s));
       };
+      ok = __all_sync(0xffffffffu, ok);
       if (ok && b >= 0) {
-        if ((ok = mbar_wait(smem_u32(&bar_kfull), 0, status, kWaitTmaFull))) {
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull), 0, status, kWaitTmaFull));
+        if (ok) {
           tc_fence_after_sync();
           issue_qk();
         }
@@ -318,20 +321,23 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       for (int j = 0; ok && b >= 0; ++j) {
         const uint32_t ph = j & 1;
         const int b_next = next_block(mrow, b, i);     // global-memory latency hidden behind the softmax
-        if (!(ok = mbar_wait(smem_u32(&bar_vfull), ph, status, kWaitTmaFull))) break;
-        if (!(ok = mbar_wait(smem_u32(&bar_p), ph, status, kWaitPReady))) break;    // P columns of keys 0..63
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_vfull), ph, status, kWaitTmaFull) &&
+                                         mbar_wait(smem_u32(&bar_p), ph, status, kWaitPReady));   // P of keys 0..63
+        if (!ok) break;
         tc_fence_after_sync();
 #pragma unroll
         for (int k16 = 0; k16 < 4; ++k16)
-          mma_ts(tmem_o, tmem_s + k16 * 8, dv + static_cast<uint64_t>((k16 * 2048) >> 4), kIdescPV, (j | k16) != 0);
-        if (!(ok = mbar_wait(smem_u32(&bar_p1), ph, status, kWaitPReady))) break;   // keys 64..127
+          mma_ts_elect(tmem_o, tmem_s + k16 * 8, dv + static_cast<uint64_t>((k16 * 2048) >> 4), kIdescPV, (j | k16) != 0);
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_p1), ph, status, kWaitPReady));         // keys 64..127
+        if (!ok) break;
         tc_fence_after_sync();
 #pragma unroll
         for (int k16 = 4; k16 < 8; ++k16)
-          mma_ts(tmem_o, tmem_s + k16 * 8, dv + static_cast<uint64_t>((k16 * 2048) >> 4), kIdescPV, 1);
-        mma_commit(smem_u32(&bar_pv));
+          mma_ts_elect(tmem_o, tmem_s + k16 * 8, dv + static_cast<uint64_t>((k16 * 2048) >> 4), kIdescPV, 1);
+        mma_commit_elect(smem_u32(&bar_pv));
         if (b_next >= 0) {                              // K of the next block arrived while the softmax ran
-          if (!(ok = mbar_wait(smem_u32(&bar_kfull), ph ^ 1, status, kWaitTmaFull))) break;
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull), ph ^ 1, status, kWaitTmaFull));
+          if (!ok) break;
           tc_fence_after_sync();
           issue_qk();
         }
