@@ -302,14 +302,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       const uint64_t dq = smem_desc_sw128(smem_u32(sQ), 16, 1024);
       const uint64_t dk = smem_desc_sw128(smem_u32(sK), 16, 1024);
       const uint64_t dv = smem_desc_sw128(smem_u32(sV), kPanel, 1024);
-      auto issue_qk = [&]() {
-#pragma unroll
-        for (int k16 = 0; k16 < 8; ++k16) {
-          const uint64_t off = static_cast<uint64_t>(((k16 >> 2) * kPanel + (k16 & 3) * 32) >> 4);
-          mma_ss_elect(tmem_s, dq + off, dk + off, kIdescQK, k16 != 0);
-        }
-        mma_commit_elect(smem_u32(&bar_s));
-      };
+      auto issue_qk = [&]() { mma_ss_k128_commit_elect(tmem_s, dq, dk, kIdescQK, kPanel, smem_u32(&bar_s)); };
       ok = __all_sync(0xffffffffu, ok);
       if (ok && b >= 0) {
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull), 0, status, kWaitTmaFull));
@@ -325,16 +318,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                                          mbar_wait(smem_u32(&bar_p), ph, status, kWaitPReady));   // P of keys 0..63
         if (!ok) break;
         tc_fence_after_sync();
-#pragma unroll
-        for (int k16 = 0; k16 < 4; ++k16)
-          mma_ts_elect(tmem_o, tmem_s + k16 * 8, dv + static_cast<uint64_t>((k16 * 2048) >> 4), kIdescPV, (j | k16) != 0);
+        mma_ts_k64_elect(tmem_o, tmem_s, dv, kIdescPV, 2048 >> 4, j != 0, 0);
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_p1), ph, status, kWaitPReady));         // keys 64..127
         if (!ok) break;
         tc_fence_after_sync();
-#pragma unroll
-        for (int k16 = 4; k16 < 8; ++k16)
-          mma_ts_elect(tmem_o, tmem_s + k16 * 8, dv + static_cast<uint64_t>((k16 * 2048) >> 4), kIdescPV, 1);
-        mma_commit_elect(smem_u32(&bar_pv));
+        mma_ts_k64_elect(tmem_o, tmem_s + 32, dv + static_cast<uint64_t>((4 * 2048) >> 4), kIdescPV, 2048 >> 4, 1, smem_u32(&bar_pv));
         if (b_next >= 0) {                              // K of the next block arrived while the softmax ran
           ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull), ph ^ 1, status, kWaitTmaFull));
           if (!ok) break;

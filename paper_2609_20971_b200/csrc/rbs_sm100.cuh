@@ -170,6 +170,58 @@ __device__ __forceinline__ void mma_commit_elect(uint32_t bar) {
       "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
       ::"r"(bar) : "memory");
 }
+// Batched issue by a converged warp: one election, then the MMAs of a whole step back to back and the commit.
+// S[d_tmem] = A B^T over K = 128 for two K-major operands stored as two 64-column panels `panel` bytes apart
+// (8 MMAs of K = 16; descriptor address field advances by 32 bytes per step inside a panel).
+__device__ __forceinline__ void mma_ss_k128_commit_elect(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                                         uint32_t panel_bytes, uint32_t bar) {
+  const uint64_t pstep = static_cast<uint64_t>(panel_bytes >> 4);
+  asm volatile(
+      "{\n\t.reg .pred e, pt, pf;\n\t.reg .b64 a, b, a1, b1;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\t"
+      "setp.eq.u32 pt, 0, 0;\n\t"
+      "setp.ne.u32 pf, 0, 0;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, pf;\n\t"
+      "add.u64 a, %1, 2;\n\t add.u64 b, %2, 2;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, pt;\n\t"
+      "add.u64 a, %1, 4;\n\t add.u64 b, %2, 4;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, pt;\n\t"
+      "add.u64 a, %1, 6;\n\t add.u64 b, %2, 6;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, pt;\n\t"
+      "add.u64 a1, %1, %4;\n\t add.u64 b1, %2, %4;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a1, b1, %3, pt;\n\t"
+      "add.u64 a, a1, 2;\n\t add.u64 b, b1, 2;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, pt;\n\t"
+      "add.u64 a, a1, 4;\n\t add.u64 b, b1, 4;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, pt;\n\t"
+      "add.u64 a, a1, 6;\n\t add.u64 b, b1, 6;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, pt;\n\t"
+      "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%5];\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "l"(pstep), "r"(bar) : "memory");
+}
+// O[d_tmem] (+)= P V for 64 keys: A = P from tensor memory (8 columns per K = 16 step from a_tmem), B = V as an
+// MN-major operand whose descriptor advances by `kstep16` (in 16-byte units) per step.  4 MMAs; the first one
+// overwrites the accumulator when `accumulate_first` is 0.  `bar` != 0: commit to that mbarrier afterwards.
+__device__ __forceinline__ void mma_ts_k64_elect(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc,
+                                                 uint32_t kstep16, uint32_t accumulate_first, uint32_t bar) {
+  const uint64_t ks = static_cast<uint64_t>(kstep16);
+  asm volatile(
+      "{\n\t.reg .pred e, pt, p0, c;\n\t.reg .b64 b;\n\t.reg .b32 a;\n\t"
+      "elect.sync _|e, 0xffffffff;\n\t"
+      "setp.eq.u32 pt, 0, 0;\n\t"
+      "setp.ne.u32 p0, %5, 0;\n\t"
+      "setp.ne.u32 c, %6, 0;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p0;\n\t"
+      "add.u32 a, %1, 8;\n\t add.u64 b, %2, %4;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, pt;\n\t"
+      "add.u32 a, %1, 16;\n\t add.u64 b, b, %4;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, pt;\n\t"
+      "add.u32 a, %1, 24;\n\t add.u64 b, b, %4;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f16 [%0], [a], b, %3, pt;\n\t"
+      "and.pred c, c, e;\n\t"
+      "@c tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%6];\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "l"(ks), "r"(accumulate_first), "r"(bar) : "memory");
+}
 // D[tmem] (+)= A[smem] * B[smem]; one thread issues.
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
