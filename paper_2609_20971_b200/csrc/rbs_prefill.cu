@@ -321,10 +321,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           issue_qk(0);
         }
       }
+      int b_next = b >= 0 ? next_block(mrow, b, i) : -1;
       for (int j = 0; ok && b >= 0; ++j) {
         const uint32_t ph = j & 1;
         const int st = j % kStages;
-        const int b_next = next_block(mrow, b, i);
+        // block index two steps ahead: its global-memory latency is hidden behind this step's waits
+        const int b_next2 = b_next >= 0 ? next_block(mrow, b_next, i) : -1;
         if (b_next >= 0) {   // S of the next block, computed under the softmax of this one
           const int sn = (j + 1) % kStages;
           ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull[sn]), ((j + 1) / kStages) & 1, status, kWaitTmaFull));
@@ -346,6 +348,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                          smem_u32(&bar_pv));
         mma_commit_elect(smem_u32(&bar_vfree[st]));
         b = b_next;
+        b_next = b_next2;
       }
     }
     __syncwarp();
@@ -359,7 +362,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     bool ok = true;
     int j = 0;
     const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
-    for (; b >= 0; ++j, b = next_block(mrow, b, i)) {
+    int b_next = b >= 0 ? next_block(mrow, b, i) : -1;
+    for (; b >= 0; ++j, b = b_next, b_next = (b_next >= 0 ? next_block(mrow, b_next, i) : -1)) {
       const uint32_t tmem_s = tmem_s0 + (j & 1) * 128;
       if (!(ok = mbar_wait(smem_u32(&bar_s[j & 1]), (j >> 1) & 1, status, kWaitMmaDone))) break;
       tc_fence_after_sync();
