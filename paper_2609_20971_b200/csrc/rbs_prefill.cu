@@ -214,24 +214,21 @@ prefill_mma_kernel(const PrefillParams p) {
 // Tensor-core path for B = 128: TMA-fed, tcgen05.mma with the accumulators in tensor memory.
 //   S[128 q x 128 keys] = Q_i K_b^T          (both operands from shared memory, 8 MMAs of K = 16)
 //   O[128 q x 128 d]   += P V_b              (P from tensor memory, V_b from shared memory, 8 MMAs)
-// One CTA per (batch, query head, query block), one CTA per SM.  S is double-buffered in tensor memory, so the
-// tensor core computes S of block j+1 while the softmax warps work on block j, and O += P V of block j while
-// they work on block j+1: in steady state the softmax warps never wait.  K and V blocks stream through
-// kStages shared-memory stages each.
-// TMEM columns: [0,128) S of even blocks, [128,256) S of odd blocks, [256,384) O.  P (bf16 pairs) is written over
-// the first 64 columns of the S buffer it came from once the owning thread has read its S row.
+// One CTA per (batch, query head, query block), two CTAs per SM so that one CTA's softmax overlaps the
+// other's matrix multiplies.  TMEM columns: [0,128) S, with P (bf16 pairs) written over [0,64) once a
+// thread has read its S row; [128,256) O.
 // Warps 0-3: softmax, one query row per thread (TMEM lane = row).  Warp 4: TMA producer.  Warp 5: MMA issuer.
+// Warps 6-7 only exist so that warps 4-7 form a whole warpgroup that can hand its registers to the softmax warps.
 // The running row maximum is only raised when a block exceeds it by more than kRescaleSlack (log2 units);
 // P then stays below 2^kRescaleSlack and O is rescaled rarely.
 // ---------------------------------------------------------------------------------------------
-constexpr int kPfThreads = 192;
-constexpr int kStages = 3;
+constexpr int kPfThreads = 256;
 constexpr float kRescaleSlack = 8.0f;
 // Of every (kPolyEvery + 1) groups of four logits, one pair is exponentiated by polynomial (0: every group
 // = 50 % of the exps, 1: 25 %, 3: 12.5 %).
 constexpr int kPolyEvery = 1;
 
-__global__ void __launch_bounds__(kPfThreads, 1)
+__global__ void __launch_bounds__(kPfThreads, 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const PrefillParams p, unsigned int* status) {
   constexpr int B = 128;
@@ -241,10 +238,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   constexpr uint32_t kIdescPV = idesc_bf16_f32(128, 128, true);
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* sQ = smem;
-  unsigned char* sK = smem + kTile;                    // kStages tiles
-  unsigned char* sV = smem + (1 + kStages) * kTile;    // kStages tiles
-  __shared__ __align__(8) uint64_t bar_q, bar_kfull[kStages], bar_kfree[kStages], bar_vfull[kStages], bar_vfree[kStages];
-  __shared__ __align__(8) uint64_t bar_s[2], bar_p, bar_p1, bar_pv;
+  unsigned char* sK = smem + kTile;
+  unsigned char* sV = smem + 2 * kTile;
+  __shared__ __align__(8) uint64_t bar_q, bar_kfull, bar_vfull, bar_s, bar_p, bar_p1, bar_pv;
   __shared__ uint32_t s_tmem;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -256,26 +252,24 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
   if (tid == 0) {
     mbar_init(smem_u32(&bar_q), 1);
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(smem_u32(&bar_kfull[s]), 1);
-      mbar_init(smem_u32(&bar_kfree[s]), 1);
-      mbar_init(smem_u32(&bar_vfull[s]), 1);
-      mbar_init(smem_u32(&bar_vfree[s]), 1);
-    }
-    mbar_init(smem_u32(&bar_s[0]), 1);
-    mbar_init(smem_u32(&bar_s[1]), 1);
+    mbar_init(smem_u32(&bar_kfull), 1);
+    mbar_init(smem_u32(&bar_vfull), 1);
+    mbar_init(smem_u32(&bar_s), 1);
     mbar_init(smem_u32(&bar_p), 128);
     mbar_init(smem_u32(&bar_p1), 128);
     mbar_init(smem_u32(&bar_pv), 1);
     mbar_fence_init();
   }
-  if (warp == 5) tmem_alloc(smem_u32(&s_tmem), 512);
+  if (warp == 5) tmem_alloc(smem_u32(&s_tmem), 256);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  const uint32_t tmem_s0 = s_tmem, tmem_o = s_tmem + 256;
+  const uint32_t tmem_s = s_tmem, tmem_o = s_tmem + 128;
 
-  if (warp == 4) {
+  if (warp >= 4) reg_dealloc<48>();
+  if (warp >= 6) {
+    // idle: registers donated above
+  } else if (warp == 4) {
     // ------------------------------- TMA producer -------------------------------
     if (lane == 0) {
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
@@ -286,74 +280,62 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         tma_load_4d(smem_u32(sQ + kPanel), &tmQ, smem_u32(&bar_q), 64, h, i * B, l);
       }
       for (int j = 0; b >= 0; ++j, b = next_block(mrow, b, i)) {
-        const int st = j % kStages, use = j / kStages;
-        if (use > 0 && !mbar_wait(smem_u32(&bar_kfree[st]), (use - 1) & 1, status, kWaitStageFree)) break;
-        mbar_arrive_expect_tx(smem_u32(&bar_kfull[st]), kTile);
-        tma_load_4d(smem_u32(sK + st * kTile), &tmK, smem_u32(&bar_kfull[st]), 0, hk, b * B, l);
-        tma_load_4d(smem_u32(sK + st * kTile + kPanel), &tmK, smem_u32(&bar_kfull[st]), 64, hk, b * B, l);
-        if (use > 0 && !mbar_wait(smem_u32(&bar_vfree[st]), (use - 1) & 1, status, kWaitStageFree)) break;
-        mbar_arrive_expect_tx(smem_u32(&bar_vfull[st]), kTile);
-        tma_load_4d(smem_u32(sV + st * kTile), &tmV, smem_u32(&bar_vfull[st]), 0, hk, b * B, l);
-        tma_load_4d(smem_u32(sV + st * kTile + kPanel), &tmV, smem_u32(&bar_vfull[st]), 64, hk, b * B, l);
+        if (j > 0 && !mbar_wait(smem_u32(&bar_s), (j - 1) & 1, status, kWaitStageFree)) break;   // S_{j-1} done: K free
+        mbar_arrive_expect_tx(smem_u32(&bar_kfull), kTile);
+        tma_load_4d(smem_u32(sK), &tmK, smem_u32(&bar_kfull), 0, hk, b * B, l);
+        tma_load_4d(smem_u32(sK + kPanel), &tmK, smem_u32(&bar_kfull), 64, hk, b * B, l);
+        if (j > 0 && !mbar_wait(smem_u32(&bar_pv), (j - 1) & 1, status, kWaitStageFree)) break;  // O_{j-1} done: V free
+        mbar_arrive_expect_tx(smem_u32(&bar_vfull), kTile);
+        tma_load_4d(smem_u32(sV), &tmV, smem_u32(&bar_vfull), 0, hk, b * B, l);
+        tma_load_4d(smem_u32(sV + kPanel), &tmV, smem_u32(&bar_vfull), 64, hk, b * B, l);
       }
     }
   } else if (warp == 5) {
     // ------------------------------- MMA issuer -------------------------------
-    // The whole warp runs this loop in lock step; one elected lane issues the tcgen05 instructions of a step in
-    // one go.  Issue order: S(0), then per block j: S(j+1), O += P(j) V(j).
+    // The whole warp runs this loop in lock step and one elected lane issues each tcgen05 instruction.
+    // Everything between two waits sits on the critical path of the tile, so the operand descriptors are
+    // built once (they only differ in the address field) and the next block index is fetched from the
+    // mask while the softmax of the current block runs.
     {
       int b = next_block(mrow, -1, i);
       bool ok = b < 0 || mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
       const uint64_t dq = smem_desc_sw128(smem_u32(sQ), 16, 1024);
       const uint64_t dk = smem_desc_sw128(smem_u32(sK), 16, 1024);
       const uint64_t dv = smem_desc_sw128(smem_u32(sV), kPanel, 1024);
-      auto issue_qk = [&](int jj) {   // S of block jj into S buffer jj & 1; frees its K stage when done
-        const int st = jj % kStages;
-        mma_ss_k128_commit_elect(tmem_s0 + (jj & 1) * 128, dq, dk + static_cast<uint64_t>((st * kTile) >> 4), kIdescQK,
-                                 kPanel, smem_u32(&bar_s[jj & 1]));
-        mma_commit_elect(smem_u32(&bar_kfree[st]));
-      };
+      auto issue_qk = [&]() { mma_ss_k128_commit_elect(tmem_s, dq, dk, kIdescQK, kPanel, smem_u32(&bar_s)); };
       ok = __all_sync(0xffffffffu, ok);
       if (ok && b >= 0) {
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull[0]), 0, status, kWaitTmaFull));
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull), 0, status, kWaitTmaFull));
         if (ok) {
           tc_fence_after_sync();
-          issue_qk(0);
+          issue_qk();
         }
       }
-      int b_next = b >= 0 ? next_block(mrow, b, i) : -1;
       for (int j = 0; ok && b >= 0; ++j) {
         const uint32_t ph = j & 1;
-        const int st = j % kStages;
-        // block index two steps ahead: its global-memory latency is hidden behind this step's waits
-        const int b_next2 = b_next >= 0 ? next_block(mrow, b_next, i) : -1;
-        if (b_next >= 0) {   // S of the next block, computed under the softmax of this one
-          const int sn = (j + 1) % kStages;
-          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull[sn]), ((j + 1) / kStages) & 1, status, kWaitTmaFull));
-          if (!ok) break;
-          tc_fence_after_sync();
-          issue_qk(j + 1);
-        }
-        const uint32_t tmem_p = tmem_s0 + ph * 128;
-        const uint64_t dvj = dv + static_cast<uint64_t>((st * kTile) >> 4);
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_vfull[st]), (j / kStages) & 1, status, kWaitTmaFull) &&
+        const int b_next = next_block(mrow, b, i);     // global-memory latency hidden behind the softmax
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_vfull), ph, status, kWaitTmaFull) &&
                                          mbar_wait(smem_u32(&bar_p), ph, status, kWaitPReady));   // P of keys 0..63
         if (!ok) break;
         tc_fence_after_sync();
-        mma_ts_k64_elect(tmem_o, tmem_p, dvj, kIdescPV, 2048 >> 4, j != 0, 0);
+        mma_ts_k64_elect(tmem_o, tmem_s, dv, kIdescPV, 2048 >> 4, j != 0, 0);
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_p1), ph, status, kWaitPReady));         // keys 64..127
         if (!ok) break;
         tc_fence_after_sync();
-        mma_ts_k64_elect(tmem_o, tmem_p + 32, dvj + static_cast<uint64_t>((4 * 2048) >> 4), kIdescPV, 2048 >> 4, 1,
-                         smem_u32(&bar_pv));
-        mma_commit_elect(smem_u32(&bar_vfree[st]));
+        mma_ts_k64_elect(tmem_o, tmem_s + 32, dv + static_cast<uint64_t>((4 * 2048) >> 4), kIdescPV, 2048 >> 4, 1, smem_u32(&bar_pv));
+        if (b_next >= 0) {                              // K of the next block arrived while the softmax ran
+          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull), ph ^ 1, status, kWaitTmaFull));
+          if (!ok) break;
+          tc_fence_after_sync();
+          issue_qk();
+        }
         b = b_next;
-        b_next = b_next2;
       }
     }
     __syncwarp();
   } else {
     // ------------------------------- softmax: one query row per thread -------------------------------
+    reg_alloc<208>();
     const int row = warp * 32 + lane;
     const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
     float m_used = -INFINITY, l_sum = 0.f;   // m_used in log2 units of the scaled logits
@@ -362,10 +344,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     bool ok = true;
     int j = 0;
     const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
-    int b_next = b >= 0 ? next_block(mrow, b, i) : -1;
-    for (; b >= 0; ++j, b = b_next, b_next = (b_next >= 0 ? next_block(mrow, b_next, i) : -1)) {
-      const uint32_t tmem_s = tmem_s0 + (j & 1) * 128;
-      if (!(ok = mbar_wait(smem_u32(&bar_s[j & 1]), (j >> 1) & 1, status, kWaitMmaDone))) break;
+    for (; b >= 0; ++j, b = next_block(mrow, b, i)) {
+      if (!(ok = mbar_wait(smem_u32(&bar_s), j & 1, status, kWaitMmaDone))) break;
       tc_fence_after_sync();
       uint32_t s[128];   // the whole S row of this thread
       {
@@ -411,7 +391,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
             for (int q = 0; q < 32; ++q) r[q] = __float_as_uint(__uint_as_float(r[q]) * corr);
             tmem_st32(tmem_o + lane_off + c0, r);
           }
-          tmem_wait_st();
         }
       }
       const uint64_t negm2 = f2_pack(-m_used, -m_used);
@@ -481,7 +460,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  if (warp == 5) tmem_dealloc(s_tmem, 512);
+  if (warp == 5) tmem_dealloc(s_tmem, 256);
 }
 
 static rbs_status launch_prefill_tc(const PrefillParams& p, const rbs_tensor& Q, const rbs_tensor& K,
@@ -493,7 +472,7 @@ static rbs_status launch_prefill_tc(const PrefillParams& p, const rbs_tensor& Q,
   if ((st = make_tmap_lthd(&tmV, V.ptr, p.L, p.N, Hkv, kHeadDim, V.stride_batch, V.stride_token, V.stride_head, 64, 128, true)) != RBS_OK) return st;
   unsigned int* status = device_status_ptr();
   if (status == nullptr) return RBS_ERR_CUDA;
-  const size_t smem = static_cast<size_t>(1 + 2 * kStages) * 2 * 128 * 128;
+  const size_t smem = 3 * 2 * 128 * 128;
   RBS_CUDA_OK(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.M;
   if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
