@@ -302,7 +302,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       const uint64_t dq = smem_desc_sw128(smem_u32(sQ), 16, 1024);
       const uint64_t dk = smem_desc_sw128(smem_u32(sK), 16, 1024);
       const uint64_t dv = smem_desc_sw128(smem_u32(sV), kPanel, 1024);
-      auto issue_qk = [&]() { mma_ss_k128_commit_elect(tmem_s, dq, dk, kIdescQK, kPanel, smem_u32(&bar_s)); };
+      auto issue_qk = [&]() { mma_ss_k128_commit_elect(tmem_s, dq, dk, kIdescQK, kPanel, kPanel, smem_u32(&bar_s)); };
       ok = __all_sync(0xffffffffu, ok);
       if (ok && b >= 0) {
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull), 0, status, kWaitTmaFull));

@@ -69,12 +69,13 @@ rescue_coeff_kernel(const float* __restrict__ radius, int M, int P /* pow2 >= M 
 // 2. fp32 centroid -> bf16 hi + bf16 lo, rows padded to Mpad with zeros
 // ---------------------------------------------------------------------------------------------
 __global__ void split_centroid_kernel(const float* __restrict__ centroid, int M, int Mpad, int64_t n_rows_padded,
-                                      __nv_bfloat16* __restrict__ chi, __nv_bfloat16* __restrict__ clo) {
-  // one thread per 4 elements
+                                      __nv_bfloat16* __restrict__ chi, __nv_bfloat16* __restrict__ clo,
+                                      float* __restrict__ cnorm) {
+  // one thread per 4 elements, one warp per centroid row (also writes the row's L2 norm)
   const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   const int64_t row = t / (kHeadDim / 4);
   const int c4 = static_cast<int>(t % (kHeadDim / 4));
-  if (row >= n_rows_padded) return;
+  if (row >= n_rows_padded) return;   // whole warps: the grid covers rows in units of 32 threads
   const int64_t hd = row / Mpad;
   const int b = static_cast<int>(row % Mpad);
   float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -90,6 +91,10 @@ __global__ void split_centroid_kernel(const float* __restrict__ centroid, int M,
   lo.y = pack_bf16(l2, l3);
   *reinterpret_cast<uint2*>(chi + row * kHeadDim + c4 * 4) = hi;
   *reinterpret_cast<uint2*>(clo + row * kHeadDim + c4 * 4) = lo;
+  float n2 = v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
+  if (c4 == 0) cnorm[row] = sqrtf(n2);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -103,7 +108,7 @@ __global__ void split_centroid_kernel(const float* __restrict__ centroid, int M,
 // ---------------------------------------------------------------------------------------------
 struct SelectParams {
   const __nv_bfloat16* Q; int64_t qsb, qst, qsh;
-  const __nv_bfloat16* chi; const __nv_bfloat16* clo; const float* g;
+  const __nv_bfloat16* chi; const __nv_bfloat16* clo; const float* g; const float* cnorm;
   int M, Mpad, W, L, Hq, G;
   float scale_log2, t_base, t_rescue;  // thresholds as log2(alpha)
   int n_sink, n_local, n_recent;
@@ -127,7 +132,7 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   float* sQn = reinterpret_cast<float*>(sQ + 2 * kPanelQ);         // B
   float* sRed = sQn + B;                                           // 32
   float* sLb = sRed + 32;
-  __shared__ __align__(8) uint64_t bar_q, bar_cfull, bar_cempty, bar_tfull[2], bar_tempty[2];
+  __shared__ __align__(8) uint64_t bar_q, bar_cfull[2], bar_cempty[2], bar_tfull[2], bar_tempty[2];   // c*: [0] hi half, [1] lo half
   __shared__ uint32_t s_tmem;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -142,8 +147,7 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
   if (tid == 0) {
     mbar_init(smem_u32(&bar_q), 1);
-    mbar_init(smem_u32(&bar_cfull), 1);
-    mbar_init(smem_u32(&bar_cempty), 1);
+    for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bar_cfull[s]), 1); mbar_init(smem_u32(&bar_cempty[s]), 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(smem_u32(&bar_tfull[s]), 1); mbar_init(smem_u32(&bar_tempty[s]), 4); }
     mbar_fence_init();
   }
@@ -160,39 +164,42 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       mbar_arrive_expect_tx(smem_u32(&bar_q), 2 * kPanelQ);
       tma_load_4d(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, i * B, l);
       tma_load_4d(smem_u32(sQ + kPanelQ), &tmQ, smem_u32(&bar_q), 64, h, i * B, l);
-      const uint32_t full = smem_u32(&bar_cfull), dst = smem_u32(sC);
+      // the hi and lo halves of a centroid tile are separate pipeline slots: the hi half of the next tile is
+      // fetched as soon as this tile's hi MMAs are done, i.e. under its lo MMAs and its epilogue
+      const uint32_t dst = smem_u32(sC);
       for (int bt = 0; bt < n_tiles; ++bt) {
-        if (bt > 0 && !mbar_wait(smem_u32(&bar_cempty), (bt - 1) & 1, status, kWaitStageFree)) break;
-        mbar_arrive_expect_tx(full, kStage);
-        tma_load_2d(dst, &tmChi, full, 0, crow0 + bt * 128);
-        tma_load_2d(dst + kPanelC, &tmChi, full, 64, crow0 + bt * 128);
-        tma_load_2d(dst + 2 * kPanelC, &tmClo, full, 0, crow0 + bt * 128);
-        tma_load_2d(dst + 3 * kPanelC, &tmClo, full, 64, crow0 + bt * 128);
+        if (bt > 0 && !mbar_wait(smem_u32(&bar_cempty[0]), (bt - 1) & 1, status, kWaitStageFree)) break;
+        mbar_arrive_expect_tx(smem_u32(&bar_cfull[0]), kStage / 2);
+        tma_load_2d(dst, &tmChi, smem_u32(&bar_cfull[0]), 0, crow0 + bt * 128);
+        tma_load_2d(dst + kPanelC, &tmChi, smem_u32(&bar_cfull[0]), 64, crow0 + bt * 128);
+        if (bt > 0 && !mbar_wait(smem_u32(&bar_cempty[1]), (bt - 1) & 1, status, kWaitStageFree)) break;
+        mbar_arrive_expect_tx(smem_u32(&bar_cfull[1]), kStage / 2);
+        tma_load_2d(dst + 2 * kPanelC, &tmClo, smem_u32(&bar_cfull[1]), 0, crow0 + bt * 128);
+        tma_load_2d(dst + 3 * kPanelC, &tmClo, smem_u32(&bar_cfull[1]), 64, crow0 + bt * 128);
       }
     }
   } else if (warp == 5) {
     // ------------------------------- MMA issuer -------------------------------
-    if (lane == 0) {
-      bool ok = mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
-      const uint32_t cbase = smem_u32(sC), qbase = smem_u32(sQ);
+    // The whole warp runs the loop; one elected lane issues the 16 MMAs of a tile in one go.
+    {
+      bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull));
+      const uint64_t dchi = smem_desc_sw128(smem_u32(sC), 16, 1024);
+      const uint64_t dclo = smem_desc_sw128(smem_u32(sC) + 2 * kPanelC, 16, 1024);
+      const uint64_t dq = smem_desc_sw128(smem_u32(sQ), 16, 1024);
       for (int bt = 0; ok && bt < n_tiles; ++bt) {
         const int buf = bt & 1;
-        ok = mbar_wait(smem_u32(&bar_cfull), bt & 1, status, kWaitTmaFull);
+        ok = mbar_wait(smem_u32(&bar_cfull[0]), bt & 1, status, kWaitTmaFull);
         if (ok && bt >= 2) ok = mbar_wait(smem_u32(&bar_tempty[buf]), ((bt >> 1) - 1) & 1, status, kWaitTmemFree);
+        ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + buf * B;
-#pragma unroll
-        for (int half = 0; half < 2; ++half) {
-#pragma unroll
-          for (int k16 = 0; k16 < 8; ++k16) {
-            const uint64_t adesc = smem_desc_sw128(cbase + (2 * half + (k16 >> 2)) * kPanelC + (k16 & 3) * 32, 16, 1024);
-            const uint64_t bdesc = smem_desc_sw128(qbase + (k16 >> 2) * kPanelQ + (k16 & 3) * 32, 16, 1024);
-            mma_ss(d_tmem, adesc, bdesc, kIdesc, (half | k16) != 0);
-          }
-        }
-        mma_commit(smem_u32(&bar_cempty));
-        mma_commit(smem_u32(&bar_tfull[buf]));
+        mma_ss_k128_commit_elect(d_tmem, dchi, dq, kIdesc, kPanelC, kPanelQ, smem_u32(&bar_cempty[0]), 0);
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_cfull[1]), bt & 1, status, kWaitTmaFull));
+        if (!ok) break;
+        tc_fence_after_sync();
+        mma_ss_k128_commit_elect(d_tmem, dclo, dq, kIdesc, kPanelC, kPanelQ, smem_u32(&bar_cempty[1]), 1);
+        mma_commit_elect(smem_u32(&bar_tfull[buf]));
       }
     }
     __syncwarp();
@@ -216,6 +223,12 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       sQn[tid] = sqrtf(s2);
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps
+    // largest query norm of the block: with it, ||q|| ||c_b|| bounds every logit of block b from above
+    float qn_max = 0.f;
+#pragma unroll
+    for (int t = lane; t < B; t += 32) qn_max = fmaxf(qn_max, sQn[t]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) qn_max = fmaxf(qn_max, __shfl_xor_sync(0xffffffffu, qn_max, o));
     const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
     for (int bt = 0; ok && bt < n_tiles; ++bt) {
       const int buf = bt & 1;
@@ -226,6 +239,13 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       const float gb = p.g[crow0 + b];            // r_b beta_b, unscaled
       const uint64_t gb2 = f2_pack(gb, gb);
       const uint32_t taddr = tmem_base + buf * B + (static_cast<uint32_t>(warp * 32) << 16);
+      // Shift of the log-sum-exp.  Any value common to the block's tokens cancels; the Cauchy-Schwarz bounds
+      // ||q||max ||c_b|| (base) and ||q||max (||c_b|| + r_b beta_b) (rescue) need no pass over the logits.  They are
+      // used when small enough that no term can underflow (2^-126); otherwise the exact maxima are taken.
+      float mb = qn_max * p.cnorm[crow0 + b] * p.scale_log2 * 1.0001f;
+      float mr = fmaf(qn_max * gb, p.scale_log2 * 1.0001f, mb);
+      const bool exact_shift = !__all_sync(0xffffffffu, mr <= 60.0f);
+      if (exact_shift) {
       // pass 1: maxima of the raw logits x and of y = x + ||q|| r beta
       float mb0 = -INFINITY, mb1 = -INFINITY, mr0 = -INFINITY, mr1 = -INFINITY;
 #pragma unroll
@@ -245,7 +265,9 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           mr1 = max3(mr1, y2, y3);
         }
       }
-      const float mb = fmaxf(mb0, mb1) * p.scale_log2, mr = fmaxf(mr0, mr1) * p.scale_log2;   // log2 units
+        mb = fmaxf(mb0, mb1) * p.scale_log2;   // log2 units
+        mr = fmaxf(mr0, mr1) * p.scale_log2;
+      }
       const uint64_t nmb2 = f2_pack(-mb, -mb), nmr2 = f2_pack(-mr, -mr);
       uint64_t sb2 = 0ull, sr2 = 0ull, sb2b = 0ull, sr2b = 0ull;
 #pragma unroll
@@ -379,6 +401,7 @@ extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats
   __nv_bfloat16* chi = reinterpret_cast<__nv_bfloat16*>(wsp + ws.off_chi);
   __nv_bfloat16* clo = reinterpret_cast<__nv_bfloat16*>(wsp + ws.off_clo);
   float* g = reinterpret_cast<float*>(wsp + ws.off_g);
+  float* cnorm = reinterpret_cast<float*>(wsp + ws.off_cn);
   unsigned int* counts = reinterpret_cast<unsigned int*>(wsp + ws.off_counts);
   const float scale_log2 = kLog2e / sqrtf(static_cast<float>(x.d));
 
@@ -392,12 +415,12 @@ extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats
   RBS_CUDA_OK(cudaGetLastError());
   const int64_t rows = static_cast<int64_t>(x.L) * x.Hkv * ws.Mpad;
   const int64_t n_thr = rows * (kHeadDim / 4);
-  split_centroid_kernel<<<static_cast<unsigned>((n_thr + 255) / 256), 256, 0, s>>>(stats.centroid, x.M, ws.Mpad, rows, chi, clo);
+  split_centroid_kernel<<<static_cast<unsigned>((n_thr + 255) / 256), 256, 0, s>>>(stats.centroid, x.M, ws.Mpad, rows, chi, clo, cnorm);
   RBS_CUDA_OK(cudaGetLastError());
 
   SelectParams p;
   p.Q = static_cast<const __nv_bfloat16*>(Q.ptr); p.qsb = Q.stride_batch; p.qst = Q.stride_token; p.qsh = Q.stride_head;
-  p.chi = chi; p.clo = clo; p.g = g;
+  p.chi = chi; p.clo = clo; p.g = g; p.cnorm = cnorm;
   p.M = x.M; p.Mpad = ws.Mpad; p.W = x.W; p.L = x.L; p.Hq = x.Hq; p.G = x.G;
   p.scale_log2 = scale_log2; p.t_base = log2f(alpha_base); p.t_rescue = log2f(alpha_rescue);
   p.n_sink = n_sink; p.n_local = n_local; p.n_recent = n_recent;

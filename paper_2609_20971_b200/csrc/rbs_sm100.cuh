@@ -172,15 +172,17 @@ __device__ __forceinline__ void mma_commit_elect(uint32_t bar) {
 }
 // Batched issue by a converged warp: one election, then the MMAs of a whole step back to back and the commit.
 // S[d_tmem] = A B^T over K = 128 for two K-major operands stored as two 64-column panels `panel` bytes apart
-// (8 MMAs of K = 16; descriptor address field advances by 32 bytes per step inside a panel).
+// (8 MMAs of K = 16; descriptor address field advances by 32 bytes per step inside a panel).  The first MMA
+// overwrites the accumulator unless `accumulate_first`; `bar` != 0: commit to that mbarrier afterwards.
 __device__ __forceinline__ void mma_ss_k128_commit_elect(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                                         uint32_t panel_bytes, uint32_t bar) {
-  const uint64_t pstep = static_cast<uint64_t>(panel_bytes >> 4);
+                                                         uint32_t a_panel_bytes, uint32_t b_panel_bytes, uint32_t bar,
+                                                         uint32_t accumulate_first = 0) {
+  const uint64_t pa = static_cast<uint64_t>(a_panel_bytes >> 4), pb = static_cast<uint64_t>(b_panel_bytes >> 4);
   asm volatile(
       "{\n\t.reg .pred e, pt, pf;\n\t.reg .b64 a, b, a1, b1;\n\t"
       "elect.sync _|e, 0xffffffff;\n\t"
       "setp.eq.u32 pt, 0, 0;\n\t"
-      "setp.ne.u32 pf, 0, 0;\n\t"
+      "setp.ne.u32 pf, %7, 0;\n\t"
       "@e tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, pf;\n\t"
       "add.u64 a, %1, 2;\n\t add.u64 b, %2, 2;\n\t"
       "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, pt;\n\t"
@@ -188,7 +190,7 @@ __device__ __forceinline__ void mma_ss_k128_commit_elect(uint32_t d_tmem, uint64
       "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, pt;\n\t"
       "add.u64 a, %1, 6;\n\t add.u64 b, %2, 6;\n\t"
       "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, pt;\n\t"
-      "add.u64 a1, %1, %4;\n\t add.u64 b1, %2, %4;\n\t"
+      "add.u64 a1, %1, %4;\n\t add.u64 b1, %2, %6;\n\t"
       "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a1, b1, %3, pt;\n\t"
       "add.u64 a, a1, 2;\n\t add.u64 b, b1, 2;\n\t"
       "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, pt;\n\t"
@@ -196,8 +198,10 @@ __device__ __forceinline__ void mma_ss_k128_commit_elect(uint32_t d_tmem, uint64
       "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, pt;\n\t"
       "add.u64 a, a1, 6;\n\t add.u64 b, b1, 6;\n\t"
       "@e tcgen05.mma.cta_group::1.kind::f16 [%0], a, b, %3, pt;\n\t"
-      "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%5];\n\t}"
-      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "l"(pstep), "r"(bar) : "memory");
+      "setp.ne.u32 pf, %5, 0;\n\t"
+      "and.pred pf, pf, e;\n\t"
+      "@pf tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%5];\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "l"(pa), "r"(bar), "l"(pb), "r"(accumulate_first) : "memory");
 }
 // O[d_tmem] (+)= P V for 64 keys: A = P from tensor memory (8 columns per K = 16 step from a_tmem), B = V as an
 // MN-major operand whose descriptor advances by `kstep16` (in 16-byte units) per step.  4 MMAs; the first one
