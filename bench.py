@@ -292,6 +292,42 @@ def run_ours(args):
     barrier()
     t_dense = e0.elapsed_time(e1) / n_dense
 
+    # optional threshold sweep: the paper's three (alpha_base, alpha_rescue) pairs and pairs calibrated by
+    # bisection to realised densities of about 3 / 5 / 10 / 15 %; each timed like the main step
+    sweep = []
+    if args.sweep and rank == 0:
+        from paper_2609_20971_b200.calibrate import calibrate_on_gpu
+        pairs = [("paper default", 0.22, 0.18), ("paper alt A", 0.16, 0.24), ("paper alt B", 0.24, 0.16)]
+        for tgt in (0.03, 0.05, 0.10, 0.15):
+            ab, ar, _ = calibrate_on_gpu(Qg, stats, B, tgt, cfg.n_sink, cfg.n_local, cfg.n_recent)
+            pairs.append((f"calibrated {tgt:.0%}", ab, ar))
+        flop_pair_s = 4.0 * B * B * cfg.d
+        for name, ab, ar in pairs:
+            evs = []
+            for rep in range(4):
+                ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+                ev[0].record(stream)
+                rbs_select(Qg, stats, B, ab, ar, cfg.n_sink, cfg.n_local, cfg.n_recent, mask=mask, density=density, workspace=ws)
+                ev[1].record(stream)
+                rbs_sparse_prefill(Qg, Kg, Vg, mask, B, out=Og)
+                ev[2].record(stream)
+                if rep > 0:
+                    evs.append(ev)
+            torch.cuda.synchronize()
+            ts = statistics.mean(e[0].elapsed_time(e[1]) for e in evs)
+            ta = statistics.mean(e[1].elapsed_time(e[2]) for e in evs)
+            dn = density.float().cpu().numpy().astype(np.float64)
+            sp = float((dn * (M * (M + 1) // 2)).sum())
+            dg = float(L * cfg.Hq * M)
+            use = flop_pair_s * ((sp - dg) + dg * (B + 1) / (2.0 * B))
+            sweep.append({"name": name, "alpha_base": ab, "alpha_rescue": ar, "density": float(dn.mean()),
+                          "t_select_ms": ts, "t_sparse_ms": ta, "speedup_vs_dense": t_dense / (ts + ta),
+                          "sparse_tensor_frac": use / (ta * 1e-3) / 1e12 / peaks["tflops"],
+                          "select_plus_sparse_tensor_frac": use / ((ts + ta) * 1e-3) / 1e12 / peaks["tflops"]})
+        # leave the default thresholds' mask and density in place for the accounting below
+        rbs_select(Qg, stats, B, *sel_args, mask=mask, density=density, workspace=ws)
+        torch.cuda.synchronize()
+
     # stats pass alone over rotating K copies (K of one layer is about the size of L2)
     n_rot = 4
     Krot = [Kg] + [Kg.clone() for _ in range(n_rot - 1)]
@@ -356,6 +392,7 @@ def run_ours(args):
             "dense_tensor_frac": dense_useful / (t_dense * 1e-3) / 1e12 / peaks["tflops"],
             "stats_rotating_us": t_stats_rot * 1e3, "stats_gbs": stats_gbs, "stats_hbm_frac": stats_gbs / peaks["hbm_gbs"],
             "peaks": peaks,
+            "sweep": sweep,
         },
     }
     print(json.dumps(out))
@@ -371,6 +408,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="q30b_128k")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="also time the threshold sweep (paper pairs + calibrated densities)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
