@@ -1,0 +1,88 @@
+"""Parity at the benchmark's full size (128K tokens, 32 query / 4 KV heads, block 128) in the launch configuration
+bench.py times: the whole path runs once on the GPU and sampled outputs are recomputed one by one by the fp64 oracle
+(statistics of one KV head, complete mask rows of sampled (head, query block) pairs, attention rows of sampled tiles,
+dense rows).  Same tolerances as the small cases."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import rbs_oracle as orc
+from paper_2609_20971_b200 import rbs_block_stats, rbs_device_status, rbs_select, rbs_sparse_prefill
+from paper_2609_20971_b200.synth import make_inputs, paper_configs, to_f64
+
+pytestmark = pytest.mark.gpu
+
+
+def _row_bits(mask, l, h, i, M):
+    words = mask[l, h, i].cpu().numpy().view(np.uint32)
+    return (((words[:, None] >> np.arange(32, dtype=np.uint32)) & 1).reshape(-1)[:M]).astype(bool)
+
+
+@pytest.fixture(scope="module")
+def full():
+    cfg = paper_configs()["q30b_128k"]
+    Q, K, V = make_inputs(cfg)
+    dev = torch.device("cuda:0")
+    Qg, Kg, Vg = Q.to(dev), K.to(dev), V.to(dev)
+    stats = rbs_block_stats(Kg, cfg.B)
+    mask, dens, mb, mr = rbs_select(Qg, stats, cfg.B, cfg.alpha_base, cfg.alpha_rescue, cfg.n_sink, cfg.n_local,
+                                    cfg.n_recent, debug=True)
+    O, lse = rbs_sparse_prefill(Qg, Kg, Vg, mask, cfg.B, return_lse=True)
+    Od = rbs_sparse_prefill(Qg, Kg, Vg, None, cfg.B)
+    torch.cuda.synchronize()
+    assert rbs_device_status() == 0
+    return dict(cfg=cfg, Q=Q, K=K, V=V, stats=stats, mask=mask, dens=dens, mb=mb, mr=mr, O=O, lse=lse, Od=Od)
+
+
+def test_fullsize_stats_and_selection(full):
+    cfg = full["cfg"]
+    M, B, G = cfg.M, cfg.B, cfg.Hq // cfg.Hkv
+    rng = np.random.default_rng(5)
+    for hk in (0, cfg.Hkv - 1):
+        K64 = to_f64(full["K"][0, :, hk])
+        c, r = orc.block_stats(K64, B)
+        beta, lo, hi = orc.rescue_coefficient(r)
+        st = full["stats"]
+        assert np.allclose(st.centroid[0, hk].cpu().numpy(), c, rtol=2e-5, atol=2e-6)
+        assert np.allclose(st.radius[0, hk].cpu().numpy(), r, rtol=2e-5)
+        assert np.allclose(st.rq[0, hk].cpu().numpy(), [lo, hi], rtol=5e-5)
+        assert np.allclose(st.beta[0, hk].cpu().numpy(), beta, atol=2e-4)
+        h = hk * G + int(rng.integers(0, G))
+        rows = sorted({0, 1, 127, 128, M - 1, M - 2} | {int(x) for x in rng.integers(0, M, size=10)})
+        sel = orc.select_head(to_f64(full["Q"][0, :, h]), c, r, beta, B, cfg.alpha_base, cfg.alpha_rescue,
+                              cfg.n_sink, cfg.n_local, cfg.n_recent, rows=rows)
+        for i in rows:
+            near_b, near_r = sel.margin_base[i] <= 1e-3, sel.margin_rescue[i] <= 1e-3
+            assert not ((_row_bits(full["mb"], 0, h, i, M) != sel.base[i]) & ~near_b).any()
+            assert not ((_row_bits(full["mr"], 0, h, i, M) != sel.rescue[i]) & ~near_r).any()
+            got = _row_bits(full["mask"], 0, h, i, M)
+            assert not ((got != sel.final[i]) & ~(near_b | near_r)).any()
+            assert not got[i + 1:].any() and got[i] and got[0]
+    # density bookkeeping over the whole mask: popcount of every head's words
+    words = full["mask"].cpu().numpy().view(np.uint32)
+    pop = np.unpackbits(words.view(np.uint8)).reshape(1, cfg.Hq, -1).sum(-1)
+    assert np.array_equal(full["dens"].cpu().numpy(), (pop / (M * (M + 1) / 2)).astype(np.float32))
+
+
+def test_fullsize_attention_rows(full):
+    cfg = full["cfg"]
+    M, B, G = cfg.M, cfg.B, cfg.Hq // cfg.Hkv
+    rng = np.random.default_rng(6)
+    got, want, got_l, want_l = [], [], [], []
+    for h in (0, 13, cfg.Hq - 1):
+        hk = h // G
+        Q64, K64, V64 = to_f64(full["Q"][0, :, h]), to_f64(full["K"][0, :, hk]), to_f64(full["V"][0, :, hk])
+        for i in sorted({0, 1, M - 1} | {int(x) for x in rng.integers(2, M - 1, size=4)}):
+            bits = _row_bits(full["mask"], 0, h, i, M)
+            o, l = orc.masked_attention_block(Q64, K64, V64, bits, i, B)
+            want.append(o); want_l.append(l)
+            got.append(full["O"][0, i * B:(i + 1) * B, h].float().cpu().numpy())
+            got_l.append(full["lse"][0, h, i * B:(i + 1) * B].cpu().numpy())
+        # one dense row in the middle of the sequence
+        i = M // 2 + h
+        o, _ = orc.masked_attention_block(Q64, K64, V64, np.ones(M, bool), i, B)
+        err = np.abs(full["Od"][0, i * B:(i + 1) * B, h].float().cpu().numpy() - o)
+        assert err.max() <= 2e-2 and err.mean() <= 2e-3
+    err = np.abs(np.concatenate(got) - np.concatenate(want))
+    assert err.max() <= 2e-2 and err.mean() <= 2e-3, (err.max(), err.mean())
+    assert np.allclose(np.concatenate(got_l), np.concatenate(want_l), atol=2e-3, rtol=1e-4)
