@@ -20,7 +20,7 @@
  *     independent problem.
  *   - Notation: N = seqlen, B = block, M = N / B blocks, Hq / Hkv query / KV heads,
  *     G = Hq / Hkv, query head h reads KV head h / G, d = head_dim, W = ceil(M / 32).
- *   - Supported: head_dim == 128, block in {64, 128}, seqlen a positive multiple of block,
+ *   - Supported: head_dim == 128, block in {64, 128, 256}, seqlen a positive multiple of block,
  *     Hq a multiple of Hkv, M <= 8192.  Anything else returns RBS_ERR_UNSUPPORTED.
  */
 #ifndef RBS_H_

@@ -8,7 +8,7 @@ rbs_status check_shape(const rbs_shape* s) {
   if (s->batch <= 0 || s->seqlen <= 0 || s->n_q_heads <= 0 || s->n_kv_heads <= 0 || s->block <= 0)
     return RBS_ERR_INVALID_ARG;
   if (s->head_dim != kHeadDim) return RBS_ERR_UNSUPPORTED;
-  if (s->block != 64 && s->block != 128) return RBS_ERR_UNSUPPORTED;
+  if (s->block != 64 && s->block != 128 && s->block != 256) return RBS_ERR_UNSUPPORTED;
   if (s->seqlen % s->block != 0) return RBS_ERR_UNSUPPORTED;
   if (s->n_q_heads % s->n_kv_heads != 0) return RBS_ERR_UNSUPPORTED;
   if (s->seqlen / s->block > 8192) return RBS_ERR_UNSUPPORTED;

@@ -14,6 +14,7 @@ struct PrefillParams {
   const uint32_t* mask;  // nullptr: dense
   float* lse;            // nullable
   int M, W, L, Hq, G, N;
+  int R;   // 128-row tiles per block (tensor-core path): block / 128
   float scale_log2;
 };
 
@@ -30,6 +31,19 @@ __device__ __forceinline__ int next_block(const uint32_t* __restrict__ row, int 
     b = (b | 31) + 1;
   }
   return -1;
+}
+
+// Tensor-core path, blocks of R x 128 tokens: the kernel works on 128-row query tiles T and 128-key sub-blocks kb.
+// Sub-block kb belongs to mask block kb / R; tile T (of query block T / R) attends sub-blocks kb <= T of the selected
+// blocks, kb == T being the diagonal one.  Returns the next sub-block after `cur` (-1 to start), or -1.
+__device__ __forceinline__ int next_kb(const uint32_t* __restrict__ row, int cur, int i, int R, int T) {
+  int kb = cur + 1;
+  if (kb > T) return -1;
+  const int b = kb / R;
+  const int nb = next_block(row, b - 1, i);   // first selected block >= b
+  if (nb < 0) return -1;
+  if (nb != b) kb = nb * R;
+  return kb <= T ? kb : -1;
 }
 
 template <int B>
@@ -211,7 +225,7 @@ prefill_mma_kernel(const PrefillParams p) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// Tensor-core path for B = 128: TMA-fed, tcgen05.mma with the accumulators in tensor memory.
+// Tensor-core path for B = 128 and B = 256 (as 128-row tiles and 128-key sub-blocks): TMA-fed, tcgen05.mma with the accumulators in tensor memory.
 //   S[128 q x 128 keys] = Q_i K_b^T          (both operands from shared memory, 8 MMAs of K = 16)
 //   O[128 q x 128 d]   += P V_b              (P from tensor memory, V_b from shared memory, 8 MMAs)
 // One CTA per (batch, query head, query block), two CTAs per SM so that one CTA's softmax overlaps the
@@ -245,7 +259,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int per_i = p.L * p.Hq;
-  const int i = p.M - 1 - static_cast<int>(blockIdx.x / per_i);
+  const int R = p.R;
+  const int T = p.M * R - 1 - static_cast<int>(blockIdx.x / per_i);   // 128-row query tile, longest rows first
+  const int i = T / R;                                                   // its query block (mask row)
   const int rem = static_cast<int>(blockIdx.x % per_i);
   const int l = rem / p.Hq, h = rem % p.Hq, hk = h / p.G;
   const uint32_t* mrow = p.mask ? p.mask + ((static_cast<int64_t>(l) * p.Hq + h) * p.M + i) * p.W : nullptr;
@@ -273,13 +289,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     // ------------------------------- TMA producer -------------------------------
     if (lane == 0) {
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
-      int b = next_block(mrow, -1, i);
+      int b = next_kb(mrow, -1, i, R, T);
       if (b >= 0) {
         mbar_arrive_expect_tx(smem_u32(&bar_q), kTile);
-        tma_load_4d(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, i * B, l);
-        tma_load_4d(smem_u32(sQ + kPanel), &tmQ, smem_u32(&bar_q), 64, h, i * B, l);
+        tma_load_4d(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, T * B, l);
+        tma_load_4d(smem_u32(sQ + kPanel), &tmQ, smem_u32(&bar_q), 64, h, T * B, l);
       }
-      for (int j = 0; b >= 0; ++j, b = next_block(mrow, b, i)) {
+      for (int j = 0; b >= 0; ++j, b = next_kb(mrow, b, i, R, T)) {
         if (j > 0 && !mbar_wait(smem_u32(&bar_s), (j - 1) & 1, status, kWaitStageFree)) break;   // S_{j-1} done: K free
         mbar_arrive_expect_tx(smem_u32(&bar_kfull), kTile);
         tma_load_4d(smem_u32(sK), &tmK, smem_u32(&bar_kfull), 0, hk, b * B, l);
@@ -297,7 +313,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     // built once (they only differ in the address field) and the next block index is fetched from the
     // mask while the softmax of the current block runs.
     {
-      int b = next_block(mrow, -1, i);
+      int b = next_kb(mrow, -1, i, R, T);
       bool ok = b < 0 || mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
       const uint64_t dq = smem_desc_sw128(smem_u32(sQ), 16, 1024);
       const uint64_t dk = smem_desc_sw128(smem_u32(sK), 16, 1024);
@@ -313,7 +329,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       }
       for (int j = 0; ok && b >= 0; ++j) {
         const uint32_t ph = j & 1;
-        const int b_next = next_block(mrow, b, i);     // global-memory latency hidden behind the softmax
+        const int b_next = next_kb(mrow, b, i, R, T);     // global-memory latency hidden behind the softmax
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_vfull), ph, status, kWaitTmaFull) &&
                                          mbar_wait(smem_u32(&bar_p), ph, status, kWaitPReady));   // P of keys 0..63
         if (!ok) break;
@@ -339,12 +355,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int row = warp * 32 + lane;
     const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
     float m_used = -INFINITY, l_sum = 0.f;   // m_used in log2 units of the scaled logits
-    int b = next_block(mrow, -1, i);
+    int b = next_kb(mrow, -1, i, R, T);
     const bool any_block = b >= 0;
     bool ok = true;
     int j = 0;
     const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
-    for (; b >= 0; ++j, b = next_block(mrow, b, i)) {
+    for (; b >= 0; ++j, b = next_kb(mrow, b, i, R, T)) {
       if (!(ok = mbar_wait(smem_u32(&bar_s), j & 1, status, kWaitMmaDone))) break;
       tc_fence_after_sync();
       uint32_t s[128];   // the whole S row of this thread
@@ -359,7 +375,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         tmem_ld32(tmem_s + lane_off + 96, s3);
         tmem_wait_ld();
       }
-      if (b == i) {   // diagonal block: keys after the query are hidden
+      if (b == T) {   // diagonal sub-block: keys after the query are hidden
 #pragma unroll
         for (int c = 0; c < 128; ++c)
           if (c > row) s[c] = 0xff800000u;   // -inf
@@ -430,8 +446,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       l_sum += (a0 + a1) + (a2 + a3);
     }
     // epilogue: O / l -> bf16 -> global
-    __nv_bfloat16* orow = p.O + l * p.osb + (static_cast<int64_t>(i) * B + row) * p.ost + h * p.osh;
-    float* lse_dst = p.lse ? p.lse + (static_cast<int64_t>(l) * p.Hq + h) * p.N + i * B + row : nullptr;
+    __nv_bfloat16* orow = p.O + l * p.osb + (static_cast<int64_t>(T) * B + row) * p.ost + h * p.osh;
+    float* lse_dst = p.lse ? p.lse + (static_cast<int64_t>(l) * p.Hq + h) * p.N + T * B + row : nullptr;
     if (!any_block) {
 #pragma unroll
       for (int c = 0; c < 16; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
@@ -474,7 +490,7 @@ static rbs_status launch_prefill_tc(const PrefillParams& p, const rbs_tensor& Q,
   if (status == nullptr) return RBS_ERR_CUDA;
   const size_t smem = 3 * 2 * 128 * 128;
   RBS_CUDA_OK(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-  const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.M;
+  const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.M * p.R;
   if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
   prefill_tc_kernel<<<static_cast<unsigned>(n_cta), kPfThreads, smem, s>>>(tmQ, tmK, tmV, p, status);
   RBS_CUDA_OK(cudaGetLastError());
@@ -493,9 +509,6 @@ static rbs_status launch_prefill(const PrefillParams& p, cudaStream_t s) {
 }
 
 }  // namespace rbs
-
-static int g_prefill_variant = 1;  // 0: mma.sync, 1: tcgen05 (B = 128)
-extern "C" __attribute__((visibility("default"))) void rbs_dev_set_prefill_variant(int v) { g_prefill_variant = v; }
 
 extern "C" rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, rbs_tensor K, rbs_tensor V,
                                          const uint32_t* mask, rbs_tensor O, float* lse, float softmax_scale,
@@ -519,6 +532,7 @@ extern "C" rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, r
   const float scale = softmax_scale == 0.f ? 1.0f / sqrtf(static_cast<float>(x.d)) : softmax_scale;
   p.scale_log2 = scale * kLog2e;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (x.B == 128 && g_prefill_variant == 1) return launch_prefill_tc(p, Q, K, V, x.Hkv, s);
-  return (x.B == 128) ? launch_prefill<128>(p, s) : launch_prefill<64>(p, s);
+  p.R = x.B / 128;
+  if (x.B >= 128) return launch_prefill_tc(p, Q, K, V, x.Hkv, s);   // tensor-core path (blocks of 128 or 256)
+  return launch_prefill<64>(p, s);                                    // blocks of 64: register-softmax mma.sync path
 }

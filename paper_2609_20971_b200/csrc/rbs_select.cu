@@ -207,11 +207,11 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     // ------------------------------- epilogue: one centroid row per thread -------------------------------
     const int row = warp * 32 + lane;
     bool ok = mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
-    if (ok && tid < B) {   // raw query norms ||q_t||_2
+    for (int tok = tid; ok && tok < B; tok += 128) {   // raw query norms ||q_t||_2
       float s2 = 0.f;
 #pragma unroll
       for (int c = 0; c < 16; ++c) {
-        const uint4 v = *reinterpret_cast<const uint4*>(sQ + (c >> 3) * kPanelQ + tid * 128 + (((c & 7) ^ (tid & 7)) << 4));
+        const uint4 v = *reinterpret_cast<const uint4*>(sQ + (c >> 3) * kPanelQ + tok * 128 + (((c & 7) ^ (tok & 7)) << 4));
         const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
@@ -220,7 +220,7 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
           s2 = fmaf(c2, c2, s2);
         }
       }
-      sQn[tid] = sqrtf(s2);
+      sQn[tok] = sqrtf(s2);
     }
     asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps
     // largest query norm of the block: with it, ||q|| ||c_b|| bounds every logit of block b from above
@@ -425,7 +425,8 @@ extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats
   p.scale_log2 = scale_log2; p.t_base = log2f(alpha_base); p.t_rescue = log2f(alpha_rescue);
   p.n_sink = n_sink; p.n_local = n_local; p.n_recent = n_recent;
   p.mask = mask; p.dbg_base = dbg_base_mask; p.dbg_rescue = dbg_rescue_mask; p.counts = counts;
-  st = (x.B == 128) ? launch_select_tc<128>(p, Q, x.N, s) : launch_select_tc<64>(p, Q, x.N, s);
+  if (x.B == 256) st = launch_select_tc<256>(p, Q, x.N, s);
+  else st = (x.B == 128) ? launch_select_tc<128>(p, Q, x.N, s) : launch_select_tc<64>(p, Q, x.N, s);
   if (st != RBS_OK) return st;
   const int nh = x.L * x.Hq;
   density_kernel<<<(nh + 127) / 128, 128, 0, s>>>(counts, nh, x.M, density);

@@ -147,5 +147,6 @@ extern "C" rbs_status rbs_block_stats(const rbs_shape* shape, rbs_tensor K, rbs_
   const long long n_tiles = static_cast<long long>(x.L) * x.Hkv * x.M;
   if (n_tiles > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  if (x.B == 256) return launch_stats_warp<256, 3>(K, x, stats, s);
   return x.B == 128 ? launch_stats_warp<128, 7>(K, x, stats, s) : launch_stats_warp<64, 14>(K, x, stats, s);
 }

@@ -56,6 +56,8 @@ CASES = {
     "ragged_b64": SynthConfig("ragged_b64", N=64 * 300, Hq=2, Hkv=1, B=64, sigma=(0.1, 1.0), seed=31),
     "gqa_b128": SynthConfig("gqa_b128", L=2, N=128 * 150, Hq=4, Hkv=2, B=128, sigma=(0.1, 1.0), seed=32,
                             n_sink=2, n_local=3, n_recent=2),
+    "gqa_b256": SynthConfig("gqa_b256", N=256 * 37, Hq=4, Hkv=2, B=256, sigma=(0.1, 1.0), seed=34, n_sink=1, n_local=2,
+                            n_recent=1),
     "lognormal_b128": SynthConfig("lognormal_b128", N=128 * 40, Hq=2, Hkv=2, B=128, sigma=0.5, sigma_ln=0.5,
                                   p_needle=0.05, seed=33),
 }
@@ -208,7 +210,7 @@ def _small(B=64, M=5, Hq=2, Hkv=1, seed=40):
     return cfg, Q, K, V
 
 
-@pytest.mark.parametrize("B", [64, 128])
+@pytest.mark.parametrize("B", [64, 128, 256])
 def test_single_block_sequence(B):
     cfg, Q, K, V = _small(B=B, M=1)
     Qg, Kg, Vg = Q.cuda(), K.cuda(), V.cuda()
