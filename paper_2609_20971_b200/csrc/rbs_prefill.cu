@@ -258,12 +258,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   __shared__ uint32_t s_tmem;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int per_i = p.L * p.Hq;
+  // Tile order: one (batch, KV head) at a time, inside it longest rows first, the G query heads of the group
+  // together.  All tiles in flight then read the K/V of one KV head (64 MiB at 128K tokens), which stays in L2;
+  // with all KV heads interleaved the K/V tiles of a 128K layer (256 MiB) were re-read from DRAM many times.
   const int R = p.R;
-  const int T = p.M * R - 1 - static_cast<int>(blockIdx.x / per_i);   // 128-row query tile, longest rows first
-  const int i = T / R;                                                   // its query block (mask row)
-  const int rem = static_cast<int>(blockIdx.x % per_i);
-  const int l = rem / p.Hq, h = rem % p.Hq, hk = h / p.G;
+  const int per_kv = p.M * R * p.G;
+  const int kvid = static_cast<int>(blockIdx.x / per_kv), rem = static_cast<int>(blockIdx.x % per_kv);
+  const int Hkv = p.Hq / p.G;
+  const int l = kvid / Hkv, hk = kvid % Hkv;
+  const int T = p.M * R - 1 - rem / p.G;   // 128-row query tile
+  const int i = T / R;                      // its query block (mask row)
+  const int h = hk * p.G + rem % p.G;
   const uint32_t* mrow = p.mask ? p.mask + ((static_cast<int64_t>(l) * p.Hq + h) * p.M + i) * p.W : nullptr;
 
   if (tid == 0) {
