@@ -26,6 +26,10 @@ if ROOT not in sys.path:
 import numpy as np
 import torch
 
+# DRAM bytes (read + write) of one rbs_sparse_prefill launch from an ncu capture of that workload at the default
+# thresholds (profiles/prefill_tc_kernel_traffic_q30b_128k.md); None where no capture of that workload exists.
+NCU_TRAFFIC_BYTES = {"q30b_128k": 3362108928 + 1045613568}
+
 METRIC = "prefill_attention_ms_per_layer_128k"
 UNIT = "ms/layer"
 
@@ -374,7 +378,8 @@ def run_ours(args):
         "config": {"workload": cfg.name, "l2": "inputs larger than L2 (Q+O 2 GiB per step)", **cfg.describe()},
         "roofline": {"bound": "tensor", "kernel": "rbs_sparse_prefill", "achieved": tflops_sparse,
                      "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": tflops_sparse / peaks["tflops"],
-                     "traffic": None, "peak_source": peaks["source"],
+                     "traffic": NCU_TRAFFIC_BYTES.get(cfg.name), "algorithmic_bytes": int(2 * Qg.numel() * 2 + 2 * Kg.numel() * 2 + mask.numel() * 4),
+                     "peak_source": peaks["source"],
                      "flops_per_launch_useful": useful, "flops_per_launch_executed": executed},
         "cpu_baseline": ({"value": cpu_ms, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                           "sample": cpu_sample, "parts": cpu_parts} if cpu_ms is not None else None),
