@@ -154,7 +154,7 @@ def run_reference(args):
     vals, sample = [], ""
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        ms, sample, _ = oracle_sample_ms_per_layer(cfg, Q, K, V, n_heads=1, n_att_rows=8)
+        ms, sample, _ = oracle_sample_ms_per_layer(cfg, Q, K, V, n_heads=4, n_att_rows=48)
         vals.append(ms)
     wall = (time.perf_counter() - t0) * 1e3 / max(args.steps, 1)
     value = float(np.mean(vals))
@@ -368,7 +368,7 @@ def run_ours(args):
     cpu_ms, cpu_sample, cpu_parts = (None, None, None)
     if world == 1 and not args.no_cpu_baseline:
         cfg0 = workload(args.workload)
-        cpu_ms, cpu_sample, cpu_parts = oracle_sample_ms_per_layer(cfg0, Q, K, V, n_heads=1, n_att_rows=24)
+        cpu_ms, cpu_sample, cpu_parts = oracle_sample_ms_per_layer(cfg0, Q, K, V, n_heads=8, n_att_rows=128)
 
     value = ms_per_layer(ms_per_step, world, L)
     out = {

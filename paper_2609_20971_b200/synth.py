@@ -66,6 +66,10 @@ def paper_configs() -> dict:
         "q30b_64k": SynthConfig("q30b_64k", N=65536, Hq=32, Hkv=4, B=128, sigma=(0.1, 1.0), p_needle=0.05,
                                 sigma_ln=0.5, seed=20974),
         "q30b_128k": SynthConfig("q30b_128k", N=131072, Hq=32, Hkv=4, B=128, sigma=(0.1, 1.0), seed=20975),
+        # the Qwen3-32B layer shape, one layer at a time, for the block-size sweep
+        "q32b_128k_b64": SynthConfig("q32b_128k_b64", N=131072, Hq=64, Hkv=8, B=64, sigma=(0.1, 1.0), seed=20977),
+        "q32b_128k_b128": SynthConfig("q32b_128k_b128", N=131072, Hq=64, Hkv=8, B=128, sigma=(0.1, 1.0), seed=20977),
+        "q32b_128k_b256": SynthConfig("q32b_128k_b256", N=131072, Hq=64, Hkv=8, B=256, sigma=(0.1, 1.0), seed=20977),
         "q32b_128k_8l": SynthConfig("q32b_128k_8l", L=8, N=131072, Hq=64, Hkv=8, B=128, sigma=(0.1, 1.0),
                                     seed=20976),
     }
