@@ -127,6 +127,25 @@ RBS_API rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, rbs_
                               void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The selector variants the paper compares with in a shared backend (Sec. 4.2, the selector ablation), through
+ * the same kernels:
+ *   RBS_SELECTOR_RBS            the method itself; identical to rbs_select.
+ *   RBS_SELECTOR_CENTROID_ONLY  mean-only scoring: beta = 0 everywhere, one relative threshold alpha_base on the
+ *                               centroid score (alpha_rescue is ignored), union with the forced blocks.
+ *   RBS_SELECTOR_FULL_L2        the unattenuated bound of Eq. (full_l2_bound) as a single ranking score: beta = 1
+ *                               everywhere, one relative threshold alpha_rescue (alpha_base is ignored), union with
+ *                               the forced blocks.
+ * stats.beta receives the beta actually used; stats.rq the quantiles (computed in every variant).
+ * Everything else is as for rbs_select.
+ */
+typedef enum { RBS_SELECTOR_RBS = 0, RBS_SELECTOR_CENTROID_ONLY = 1, RBS_SELECTOR_FULL_L2 = 2 } rbs_selector;
+RBS_API rbs_status rbs_select_variant(const rbs_shape* shape, rbs_tensor Q, rbs_stats stats, rbs_selector which,
+                                      float alpha_base, float alpha_rescue, int n_sink, int n_local, int n_recent,
+                                      uint32_t* mask, float* density, uint32_t* dbg_base_mask,
+                                      uint32_t* dbg_rescue_mask, void* workspace, size_t workspace_bytes,
+                                      void* stream);
+
+/*
  * rbs_select for callers that have no device memory to hand over and must not allocate any.
  * (The paper has no counterpart: this is a packaging variant of rbs_select, same arithmetic, same outputs.)
  *

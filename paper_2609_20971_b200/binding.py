@@ -16,6 +16,7 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "librbs_b200.so")
 
 RBS_OP_BLOCK_STATS, RBS_OP_SELECT, RBS_OP_SPARSE_PREFILL = 0, 1, 2
+SELECTOR_RBS, SELECTOR_CENTROID_ONLY, SELECTOR_FULL_L2 = 0, 1, 2
 
 
 class RbsShape(ctypes.Structure):
@@ -56,6 +57,8 @@ def load_library() -> ctypes.CDLL:
     lib.rbs_block_stats.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, vp]
     lib.rbs_select.restype = i
     lib.rbs_select.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, f, f, i, i, i, vp, vp, vp, vp, vp, sz, vp]
+    lib.rbs_select_variant.restype = i
+    lib.rbs_select_variant.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, i, f, f, i, i, i, vp, vp, vp, vp, vp, sz, vp]
     lib.rbs_select_static.restype = i
     lib.rbs_select_static.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, f, f, i, i, i, vp, vp, vp, vp, vp]
     lib.rbs_sparse_prefill.restype = i
@@ -143,9 +146,11 @@ def rbs_block_stats(K: torch.Tensor, block: int, stats: BlockStats | None = None
 
 def rbs_select(Q: torch.Tensor, stats: BlockStats, block: int, alpha_base: float = 0.22, alpha_rescue: float = 0.18,
                n_sink: int = 1, n_local: int = 1, n_recent: int = 1, *, mask: torch.Tensor | None = None,
-               density: torch.Tensor | None = None, workspace: torch.Tensor | None = None, debug: bool = False):
+               density: torch.Tensor | None = None, workspace: torch.Tensor | None = None, debug: bool = False,
+               selector: int = 0):
     """Dual-branch block selection (Sec. 3.2).  Returns (mask uint32-as-int32 [L,Hq,M,W], density [L,Hq])
-    and, with debug=True, also the base and rescue branch masks."""
+    and, with debug=True, also the base and rescue branch masks.  `selector`: SELECTOR_RBS (default),
+    SELECTOR_CENTROID_ONLY or SELECTOR_FULL_L2 (the comparison selectors of the paper's ablation)."""
     lib = load_library()
     L, N, Hq, d = Q.shape
     Hkv = stats.centroid.shape[1]
@@ -162,9 +167,14 @@ def rbs_select(Q: torch.Tensor, stats: BlockStats, block: int, alpha_base: float
         workspace = torch.empty(max(need, 256), dtype=torch.uint8, device=dev)
     dbg_b = torch.empty_like(mask) if debug else None
     dbg_r = torch.empty_like(mask) if debug else None
-    _check(lib.rbs_select(ctypes.byref(shape), _tensor(Q), stats.c_struct(), alpha_base, alpha_rescue,
-                          n_sink, n_local, n_recent, _ptr(mask), _ptr(density), _ptr(dbg_b), _ptr(dbg_r),
-                          _ptr(workspace), workspace.numel(), _stream()), "rbs_select")
+    if selector == SELECTOR_RBS:
+        _check(lib.rbs_select(ctypes.byref(shape), _tensor(Q), stats.c_struct(), alpha_base, alpha_rescue,
+                              n_sink, n_local, n_recent, _ptr(mask), _ptr(density), _ptr(dbg_b), _ptr(dbg_r),
+                              _ptr(workspace), workspace.numel(), _stream()), "rbs_select")
+    else:
+        _check(lib.rbs_select_variant(ctypes.byref(shape), _tensor(Q), stats.c_struct(), selector, alpha_base,
+                                      alpha_rescue, n_sink, n_local, n_recent, _ptr(mask), _ptr(density), _ptr(dbg_b),
+                                      _ptr(dbg_r), _ptr(workspace), workspace.numel(), _stream()), "rbs_select_variant")
     if debug:
         return mask, density, dbg_b, dbg_r
     return mask, density

@@ -19,7 +19,8 @@ constexpr int kCoeffThreads = 1024;
 
 __global__ void __launch_bounds__(kCoeffThreads)
 rescue_coeff_kernel(const float* __restrict__ radius, int M, int P /* pow2 >= M */, float scale_log2,
-                    float* __restrict__ beta, float* __restrict__ rq, float* __restrict__ g, int Mpad) {
+                    float* __restrict__ beta, float* __restrict__ rq, float* __restrict__ g, int Mpad,
+                    int beta_mode /* 0: Eq. (beta), 1: beta = 0, 2: beta = 1 */) {
   extern __shared__ float s_sorted[];
   __shared__ float s_q[2];
   const int hd = blockIdx.x, tid = threadIdx.x;
@@ -59,6 +60,8 @@ rescue_coeff_kernel(const float* __restrict__ radius, int M, int P /* pow2 >= M 
     if (idx < M) {
       rb = r[idx];
       bt = live ? fminf(fmaxf((rb - r_low) * inv, 0.f), 1.f) : 0.f;
+      if (beta_mode == 1) bt = 0.f;
+      if (beta_mode == 2) bt = 1.f;
       beta[static_cast<int64_t>(hd) * M + idx] = bt;
     }
     g[static_cast<int64_t>(hd) * Mpad + idx] = rb * bt;
@@ -380,10 +383,10 @@ static rbs_status launch_select_tc(const SelectParams& p, const rbs_tensor& Q, i
 
 }  // namespace rbs
 
-extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats stats, float alpha_base,
-                                 float alpha_rescue, int n_sink, int n_local, int n_recent, uint32_t* mask,
-                                 float* density, uint32_t* dbg_base_mask, uint32_t* dbg_rescue_mask,
-                                 void* workspace, size_t workspace_bytes, void* stream) {
+static rbs_status select_impl(const rbs_shape* shape, rbs_tensor Q, rbs_stats stats, int beta_mode, float alpha_base,
+                              float alpha_rescue, int n_sink, int n_local, int n_recent, uint32_t* mask,
+                              float* density, uint32_t* dbg_base_mask, uint32_t* dbg_rescue_mask,
+                              void* workspace, size_t workspace_bytes, void* stream) {
   using namespace rbs;
   rbs_status st = check_shape(shape);
   if (st != RBS_OK) return st;
@@ -411,7 +414,7 @@ extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats
   const size_t coeff_smem = static_cast<size_t>(P) * sizeof(float);
   RBS_CUDA_OK(cudaMemsetAsync(counts, 0, static_cast<size_t>(x.L) * x.Hq * sizeof(unsigned int), s));
   rescue_coeff_kernel<<<x.L * x.Hkv, kCoeffThreads, coeff_smem, s>>>(stats.radius, x.M, P, scale_log2, stats.beta,
-                                                                     stats.rq, g, ws.Mpad);
+                                                                     stats.rq, g, ws.Mpad, beta_mode);
   RBS_CUDA_OK(cudaGetLastError());
   const int64_t rows = static_cast<int64_t>(x.L) * x.Hkv * ws.Mpad;
   const int64_t n_thr = rows * (kHeadDim / 4);
@@ -432,6 +435,34 @@ extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats
   density_kernel<<<(nh + 127) / 128, 128, 0, s>>>(counts, nh, x.M, density);
   RBS_CUDA_OK(cudaGetLastError());
   return RBS_OK;
+}
+
+extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats stats, float alpha_base,
+                                 float alpha_rescue, int n_sink, int n_local, int n_recent, uint32_t* mask,
+                                 float* density, uint32_t* dbg_base_mask, uint32_t* dbg_rescue_mask,
+                                 void* workspace, size_t workspace_bytes, void* stream) {
+  return select_impl(shape, Q, stats, 0, alpha_base, alpha_rescue, n_sink, n_local, n_recent, mask, density,
+                     dbg_base_mask, dbg_rescue_mask, workspace, workspace_bytes, stream);
+}
+
+extern "C" rbs_status rbs_select_variant(const rbs_shape* shape, rbs_tensor Q, rbs_stats stats, rbs_selector which,
+                                         float alpha_base, float alpha_rescue, int n_sink, int n_local, int n_recent,
+                                         uint32_t* mask, float* density, uint32_t* dbg_base_mask,
+                                         uint32_t* dbg_rescue_mask, void* workspace, size_t workspace_bytes,
+                                         void* stream) {
+  constexpr float kDisabled = 2.0f;   // alpha > 1 empties a branch
+  switch (which) {
+    case RBS_SELECTOR_RBS:
+      return select_impl(shape, Q, stats, 0, alpha_base, alpha_rescue, n_sink, n_local, n_recent, mask, density,
+                         dbg_base_mask, dbg_rescue_mask, workspace, workspace_bytes, stream);
+    case RBS_SELECTOR_CENTROID_ONLY:
+      return select_impl(shape, Q, stats, 1, alpha_base, kDisabled, n_sink, n_local, n_recent, mask, density,
+                         dbg_base_mask, dbg_rescue_mask, workspace, workspace_bytes, stream);
+    case RBS_SELECTOR_FULL_L2:
+      return select_impl(shape, Q, stats, 2, kDisabled, alpha_rescue, n_sink, n_local, n_recent, mask, density,
+                         dbg_base_mask, dbg_rescue_mask, workspace, workspace_bytes, stream);
+  }
+  return RBS_ERR_INVALID_ARG;
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -296,3 +296,22 @@ def test_select_is_deterministic_and_reusable_workspace():
     m1, d1 = rbs_select(Qg, stats, cfg.B)
     m2, d2 = rbs_select(Qg, stats, cfg.B)
     assert torch.equal(m1, m2) and torch.equal(d1, d2)
+
+
+def test_selector_variants_match_the_oracle_with_fixed_beta():
+    """Centroid-only (beta = 0, one threshold) and Full-L2 (beta = 1, one threshold) through rbs_select_variant."""
+    from paper_2609_20971_b200.binding import SELECTOR_CENTROID_ONLY, SELECTOR_FULL_L2
+    cfg, Q, K, V = _small(B=128, M=140, Hq=2, Hkv=1, seed=44)
+    Qg, Kg = Q.cuda(), K.cuda()
+    stats = rbs_block_stats(Kg, cfg.B)
+    Q64, K64 = to_f64(Q), to_f64(K)
+    c, r = orc.block_stats(K64[0, :, 0], cfg.B)
+    for selector, beta, ab, ar in ((SELECTOR_CENTROID_ONLY, np.zeros_like(r), 0.194, 2.0),
+                                   (SELECTOR_FULL_L2, np.ones_like(r), 2.0, 0.022)):
+        mask, dens = rbs_select(Qg, stats, cfg.B, ab if ab < 1 else 0.5, ar if ar < 1 else 0.5, 1, 1, 1, selector=selector)
+        assert np.array_equal(stats.beta.cpu().numpy()[0, 0], beta.astype(np.float32))
+        got = unpack_mask(mask, cfg.M)
+        for h in range(cfg.Hq):
+            s = orc.select_head(Q64[0, :, h], c, r, beta, cfg.B, ab, ar, 1, 1, 1)
+            near = (s.margin_base <= MASK_MARGIN) if ab < 1 else (s.margin_rescue <= MASK_MARGIN)
+            assert not ((got[0, h] != s.final) & ~near).any()
