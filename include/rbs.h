@@ -18,9 +18,9 @@
  *     (strides in elements, multiples of 8; ptr 16-byte aligned).  The natural layout is
  *     [batch][token][head][head_dim].  `batch` is prompts x layers: every (batch, KV head) is an
  *     independent problem.
- *   - Notation: N = seqlen, B = block, M = N / B blocks, Hq / Hkv query / KV heads,
+ *   - Notation: N = seqlen, B = block, M = ceil(N / B) blocks (a short last block is allowed), Hq / Hkv query / KV heads,
  *     G = Hq / Hkv, query head h reads KV head h / G, d = head_dim, W = ceil(M / 32).
- *   - Supported: head_dim == 128, block in {64, 128, 256}, seqlen a positive multiple of block,
+ *   - Supported: head_dim == 128, block in {64, 128, 256}, seqlen positive,
  *     Hq a multiple of Hkv, M <= 8192.  Anything else returns RBS_ERR_UNSUPPORTED.
  */
 #ifndef RBS_H_

@@ -159,21 +159,20 @@ def select_head(Q: np.ndarray, centroid: np.ndarray, radius: np.ndarray, beta: n
                 n_sink: int, n_local: int, n_recent: int, rows=None) -> HeadSelection:
     """Algorithm 1, third loop, for ONE query head against its KV head's statistics.
 
-    Q [N, d]; centroid [M, d]; radius, beta [M].  N must be a multiple of `block`.
+    Q [N, d]; centroid [M, d]; radius, beta [M].  A short last query block aggregates over its own tokens.
     `rows` (optional) restricts the work to those query blocks; other rows stay empty and the
     returned density is then meaningless.
     """
     Q = np.asarray(Q, dtype=np.float64)
     N, d = Q.shape
     M = n_blocks(N, block)
-    assert N == M * block, "selector oracle takes whole query blocks"
     base = np.zeros((M, M), dtype=bool)
     rescue = np.zeros((M, M), dtype=bool)
     forced = np.zeros((M, M), dtype=bool)
     margin_base = np.full((M, M), np.inf)
     margin_rescue = np.full((M, M), np.inf)
     for i in (range(M) if rows is None else rows):
-        Qi = Q[i * block:(i + 1) * block]
+        Qi = Q[i * block:min(N, (i + 1) * block)]
         nb = i + 1  # causal candidates C_i = {0..i}
         l_base, l_rescue = branch_logits(Qi, centroid[:nb], radius[:nb], beta[:nb])
         S_base = aggregate(l_base, d)

@@ -112,7 +112,7 @@ class BlockStats:
 
 def alloc_stats(K: torch.Tensor, block: int) -> BlockStats:
     L, N, Hkv, d = K.shape
-    M = N // block
+    M = (N + block - 1) // block
     dev = K.device
     return BlockStats(torch.empty(L, Hkv, M, d, dtype=torch.float32, device=dev),
                       torch.empty(L, Hkv, M, dtype=torch.float32, device=dev),
@@ -154,7 +154,7 @@ def rbs_select(Q: torch.Tensor, stats: BlockStats, block: int, alpha_base: float
     lib = load_library()
     L, N, Hq, d = Q.shape
     Hkv = stats.centroid.shape[1]
-    M = N // block
+    M = (N + block - 1) // block
     W = (M + 31) // 32
     shape = RbsShape(L, N, Hq, Hkv, d, block)
     dev = Q.device

@@ -48,7 +48,7 @@ def calibrate_on_gpu(Q, stats, block: int, target: float, n_sink: int = 1, n_loc
 
     from .binding import RBS_OP_SELECT, RbsShape, rbs_select, workspace_bytes
     L, N, Hq, d = Q.shape
-    M = N // block
+    M = (N + block - 1) // block
     shape = RbsShape(L, N, Hq, stats.centroid.shape[1], d, block)
     mask = torch.empty(L, Hq, M, (M + 31) // 32, dtype=torch.int32, device=Q.device)
     dens = torch.empty(L, Hq, dtype=torch.float32, device=Q.device)

@@ -9,9 +9,8 @@ rbs_status check_shape(const rbs_shape* s) {
     return RBS_ERR_INVALID_ARG;
   if (s->head_dim != kHeadDim) return RBS_ERR_UNSUPPORTED;
   if (s->block != 64 && s->block != 128 && s->block != 256) return RBS_ERR_UNSUPPORTED;
-  if (s->seqlen % s->block != 0) return RBS_ERR_UNSUPPORTED;
   if (s->n_q_heads % s->n_kv_heads != 0) return RBS_ERR_UNSUPPORTED;
-  if (s->seqlen / s->block > 8192) return RBS_ERR_UNSUPPORTED;
+  if ((s->seqlen + s->block - 1) / s->block > 8192) return RBS_ERR_UNSUPPORTED;
   return RBS_OK;
 }
 

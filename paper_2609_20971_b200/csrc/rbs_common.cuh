@@ -22,7 +22,7 @@ struct Dims {
 inline Dims make_dims(const rbs_shape& s) {
   Dims x;
   x.L = s.batch; x.N = s.seqlen; x.Hq = s.n_q_heads; x.Hkv = s.n_kv_heads; x.d = s.head_dim; x.B = s.block;
-  x.M = s.block > 0 ? s.seqlen / s.block : 0;
+  x.M = s.block > 0 ? (s.seqlen + s.block - 1) / s.block : 0;   // a short last block counts
   x.W = (x.M + 31) / 32;
   x.G = s.n_kv_heads > 0 ? s.n_q_heads / s.n_kv_heads : 0;
   return x;
@@ -83,6 +83,11 @@ __device__ __forceinline__ uint32_t smem_u32(const void* p) {
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src));
+}
+// 16-byte copy that writes zeros instead when `valid` is false (nothing is read from `src` then)
+__device__ __forceinline__ void cp_async16_zfill(uint32_t dst, const void* src, bool valid) {
+  const uint32_t n = valid ? 16u : 0u;
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n));
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;"); }
 template <int N>

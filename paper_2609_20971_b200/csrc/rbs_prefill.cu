@@ -73,27 +73,32 @@ prefill_mma_kernel(const PrefillParams p) {
   auto load_kv = [&](int b, int stage) {
     const __nv_bfloat16* ks = kbase + static_cast<int64_t>(b) * B * p.kst;
     const __nv_bfloat16* vs = vbase + static_cast<int64_t>(b) * B * p.vst;
+    const int rows_in = p.N - b * B;   // keys past the sequence end are loaded as zeros (and hidden by causality)
     for (int c = tid; c < B * 16; c += NTHREADS) {
       const int row = c >> 4, chunk = c & 15;
-      cp_async16(smem_u32(sK + stage * TILE + tile_off(row, chunk)), ks + static_cast<int64_t>(row) * p.kst + chunk * 8);
-      cp_async16(smem_u32(sV + stage * TILE + tile_off(row, chunk)), vs + static_cast<int64_t>(row) * p.vst + chunk * 8);
+      const bool in = row < rows_in;
+      const int64_t r = in ? row : 0;
+      cp_async16_zfill(smem_u32(sK + stage * TILE + tile_off(row, chunk)), ks + r * p.kst + chunk * 8, in);
+      cp_async16_zfill(smem_u32(sV + stage * TILE + tile_off(row, chunk)), vs + r * p.vst + chunk * 8, in);
     }
   };
 
   int b_cur = next_block(mrow, -1, i);
   const int row0 = warp * 16 + gq;  // this thread's first query row inside the block (second: +8)
+  const int q_rows = min(B, p.N - i * B);   // a short last query block: rows past the sequence end are not written
   if (b_cur < 0) {                  // nothing retained: zero rows, lse = -inf
     for (int c = tid; c < B * 16; c += NTHREADS) {
       const int row = c >> 4, chunk = c & 15;
-      *reinterpret_cast<uint4*>(obase + static_cast<int64_t>(row) * p.ost + chunk * 8) = make_uint4(0, 0, 0, 0);
+      if (row < q_rows) *reinterpret_cast<uint4*>(obase + static_cast<int64_t>(row) * p.ost + chunk * 8) = make_uint4(0, 0, 0, 0);
     }
-    if (p.lse && tid < B) p.lse[(static_cast<int64_t>(l) * p.Hq + h) * p.N + i * B + tid] = -INFINITY;
+    if (p.lse && tid < q_rows) p.lse[(static_cast<int64_t>(l) * p.Hq + h) * p.N + i * B + tid] = -INFINITY;
     return;
   }
 
   for (int c = tid; c < B * 16; c += NTHREADS) {
     const int row = c >> 4, chunk = c & 15;
-    cp_async16(smem_u32(sQ + tile_off(row, chunk)), qbase + static_cast<int64_t>(row) * p.qst + chunk * 8);
+    const bool in = row < q_rows;
+    cp_async16_zfill(smem_u32(sQ + tile_off(row, chunk)), qbase + static_cast<int64_t>(in ? row : 0) * p.qst + chunk * 8, in);
   }
   load_kv(b_cur, 0);
   cp_async_commit();
@@ -214,13 +219,13 @@ prefill_mma_kernel(const PrefillParams p) {
   __nv_bfloat16* o1 = obase + static_cast<int64_t>(row0 + 8) * p.ost;
 #pragma unroll
   for (int n = 0; n < 16; ++n) {
-    *reinterpret_cast<uint32_t*>(o0 + n * 8 + tq * 2) = pack_bf16(acc_o[n][0] * inv0, acc_o[n][1] * inv0);
-    *reinterpret_cast<uint32_t*>(o1 + n * 8 + tq * 2) = pack_bf16(acc_o[n][2] * inv1, acc_o[n][3] * inv1);
+    if (row0 < q_rows) *reinterpret_cast<uint32_t*>(o0 + n * 8 + tq * 2) = pack_bf16(acc_o[n][0] * inv0, acc_o[n][1] * inv0);
+    if (row0 + 8 < q_rows) *reinterpret_cast<uint32_t*>(o1 + n * 8 + tq * 2) = pack_bf16(acc_o[n][2] * inv1, acc_o[n][3] * inv1);
   }
   if (p.lse && tq == 0) {
     float* dst = p.lse + (static_cast<int64_t>(l) * p.Hq + h) * p.N + i * B;
-    dst[row0] = (m_run[0] + fast_log2(l_run[0])) * 0.6931471805599453f;
-    dst[row0 + 8] = (m_run[1] + fast_log2(l_run[1])) * 0.6931471805599453f;
+    if (row0 < q_rows) dst[row0] = (m_run[0] + fast_log2(l_run[0])) * 0.6931471805599453f;
+    if (row0 + 8 < q_rows) dst[row0 + 8] = (m_run[1] + fast_log2(l_run[1])) * 0.6931471805599453f;
   }
 }
 
@@ -269,6 +274,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const int T = p.M * R - 1 - rem / p.G;   // 128-row query tile
   const int i = T / R;                      // its query block (mask row)
   const int h = hk * p.G + rem % p.G;
+  if (T * 128 >= p.N) return;               // a tile wholly past the sequence end (short last block of 256)
   const uint32_t* mrow = p.mask ? p.mask + ((static_cast<int64_t>(l) * p.Hq + h) * p.M + i) * p.W : nullptr;
 
   if (tid == 0) {
@@ -453,10 +459,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     // epilogue: O / l -> bf16 -> global
     __nv_bfloat16* orow = p.O + l * p.osb + (static_cast<int64_t>(T) * B + row) * p.ost + h * p.osh;
     float* lse_dst = p.lse ? p.lse + (static_cast<int64_t>(l) * p.Hq + h) * p.N + T * B + row : nullptr;
+    const bool in_seq = T * B + row < p.N;   // rows of a short last block past the sequence end are not written
     if (!any_block) {
+      if (in_seq) {
 #pragma unroll
-      for (int c = 0; c < 16; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
-      if (lse_dst) *lse_dst = -INFINITY;
+        for (int c = 0; c < 16; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
+        if (lse_dst) *lse_dst = -INFINITY;
+      }
     } else if (ok && mbar_wait(smem_u32(&bar_pv), (j - 1) & 1, status, kWaitOReady)) {
       tc_fence_after_sync();
       const float inv = 1.0f / l_sum;
@@ -472,10 +481,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           v.y = pack_bf16(__uint_as_float(r[q + 2]) * inv, __uint_as_float(r[q + 3]) * inv);
           v.z = pack_bf16(__uint_as_float(r[q + 4]) * inv, __uint_as_float(r[q + 5]) * inv);
           v.w = pack_bf16(__uint_as_float(r[q + 6]) * inv, __uint_as_float(r[q + 7]) * inv);
-          *reinterpret_cast<uint4*>(orow + c0 + q) = v;
+          if (in_seq) *reinterpret_cast<uint4*>(orow + c0 + q) = v;
         }
       }
-      if (lse_dst) *lse_dst = (m_used + fast_log2(l_sum)) * 0.6931471805599453f;
+      if (lse_dst && in_seq) *lse_dst = (m_used + fast_log2(l_sum)) * 0.6931471805599453f;
     }
   }
   tc_fence_before_sync();

@@ -112,7 +112,7 @@ __global__ void split_centroid_kernel(const float* __restrict__ centroid, int M,
 struct SelectParams {
   const __nv_bfloat16* Q; int64_t qsb, qst, qsh;
   const __nv_bfloat16* chi; const __nv_bfloat16* clo; const float* g; const float* cnorm;
-  int M, Mpad, W, L, Hq, G;
+  int M, Mpad, W, L, Hq, G, N;
   float scale_log2, t_base, t_rescue;  // thresholds as log2(alpha)
   int n_sink, n_local, n_recent;
   uint32_t* mask; uint32_t* dbg_base; uint32_t* dbg_rescue;
@@ -233,6 +233,7 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) qn_max = fmaxf(qn_max, __shfl_xor_sync(0xffffffffu, qn_max, o));
     const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
+    const int n_tok = min(B, p.N - i * B);
     for (int bt = 0; ok && bt < n_tiles; ++bt) {
       const int buf = bt & 1;
       ok = mbar_wait(smem_u32(&bar_tfull[buf]), (bt >> 1) & 1, status, kWaitMmaDone);
@@ -256,6 +257,11 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         uint32_t r[32];
         tmem_ld32(taddr + c0, r);
         tmem_wait_ld();
+        if (n_tok < B) {   // short last query block: tokens past the sequence end do not count
+#pragma unroll
+          for (int q = 0; q < 32; ++q)
+            if (c0 + q >= n_tok) r[q] = 0xff800000u;   // -inf
+        }
 #pragma unroll
         for (int j = 0; j < 32; j += 4) {
           const float4 qn = *reinterpret_cast<const float4*>(sQn + c0 + j);
@@ -278,6 +284,11 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         uint32_t r[32];
         tmem_ld32(taddr + c0, r);
         tmem_wait_ld();
+        if (n_tok < B) {   // short last query block: tokens past the sequence end do not count
+#pragma unroll
+          for (int q = 0; q < 32; ++q)
+            if (c0 + q >= n_tok) r[q] = 0xff800000u;   // -inf
+        }
         if (c0 + 32 >= B) {   // accumulator fully read: hand the TMEM buffer back to the MMA warp
           tc_fence_before_sync();
           __syncwarp();
@@ -424,7 +435,7 @@ static rbs_status select_impl(const rbs_shape* shape, rbs_tensor Q, rbs_stats st
   SelectParams p;
   p.Q = static_cast<const __nv_bfloat16*>(Q.ptr); p.qsb = Q.stride_batch; p.qst = Q.stride_token; p.qsh = Q.stride_head;
   p.chi = chi; p.clo = clo; p.g = g; p.cnorm = cnorm;
-  p.M = x.M; p.Mpad = ws.Mpad; p.W = x.W; p.L = x.L; p.Hq = x.Hq; p.G = x.G;
+  p.M = x.M; p.Mpad = ws.Mpad; p.W = x.W; p.L = x.L; p.Hq = x.Hq; p.G = x.G; p.N = x.N;
   p.scale_log2 = scale_log2; p.t_base = log2f(alpha_base); p.t_rescue = log2f(alpha_rescue);
   p.n_sink = n_sink; p.n_local = n_local; p.n_recent = n_recent;
   p.mask = mask; p.dbg_base = dbg_base_mask; p.dbg_rescue = dbg_rescue_mask; p.counts = counts;

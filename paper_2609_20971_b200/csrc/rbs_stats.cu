@@ -15,7 +15,7 @@ namespace rbs {
 // ---------------------------------------------------------------------------------------------
 template <int B, int NW>
 __global__ void __launch_bounds__(NW * 32, 1)
-block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, int M, int Hkv,
+block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, int M, int Hkv, int N,
                         float* __restrict__ centroid, float* __restrict__ radius, unsigned int* status) {
   constexpr uint32_t kPanel = B * 128;       // bytes of one 64-column panel
   constexpr uint32_t kSlot = 2 * kPanel;
@@ -62,11 +62,14 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
         a0 += bf16lo(lo); a1 += bf16hi(lo); a2 += bf16lo(hi); a3 += bf16hi(hi);
       }
     }
-    const float4 cen = make_float4(a0 * (1.0f / B), a1 * (1.0f / B), a2 * (1.0f / B), a3 * (1.0f / B));
     int idx = t;
     const int hk = idx % Hkv; idx /= Hkv;
     const int b = idx % M;
     const int l = idx / M;
+    // a short last block: TMA filled the rows past the sequence end with zeros; divide by its own size |K_b|
+    const int rows_valid = min(B, N - b * B);
+    const float inv_rows = 1.0f / static_cast<float>(rows_valid);
+    const float4 cen = make_float4(a0 * inv_rows, a1 * inv_rows, a2 * inv_rows, a3 * inv_rows);
     const int64_t blk = (static_cast<int64_t>(l) * Hkv + hk) * M + b;
     reinterpret_cast<float4*>(centroid + blk * kHeadDim)[lane] = cen;
 
@@ -100,9 +103,10 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
         d = bf16hi(x3) - cb.w; q[j] = fmaf(d, d, q[j]);
       }
     }
-    float rmax = q[0];
+    float rmax = 0.f;
 #pragma unroll
-    for (int j = 1; j < RJ; ++j) rmax = fmaxf(rmax, q[j]);
+    for (int j = 0; j < RJ; ++j)
+      if (lane + 32 * j < rows_valid) rmax = fmaxf(rmax, q[j]);
     __syncwarp();   // every lane is done reading the slot
     if (lane == 0 && t + stride < n_tiles) {
       fence_proxy_async_smem();
@@ -128,7 +132,7 @@ static rbs_status launch_stats_warp(const rbs_tensor& K, const Dims& x, const rb
   const long long n_tiles = static_cast<long long>(x.L) * x.Hkv * x.M;
   long long want = (n_tiles + NW - 1) / NW;
   const int grid = static_cast<int>(want < sm_count() ? want : sm_count());
-  kern<<<grid, NW * 32, smem, s>>>(tm, static_cast<int>(n_tiles), x.M, x.Hkv, stats.centroid, stats.radius, status);
+  kern<<<grid, NW * 32, smem, s>>>(tm, static_cast<int>(n_tiles), x.M, x.Hkv, x.N, stats.centroid, stats.radius, status);
   RBS_CUDA_OK(cudaGetLastError());
   return RBS_OK;
 }

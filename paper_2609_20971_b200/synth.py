@@ -49,7 +49,7 @@ class SynthConfig:
 
     @property
     def M(self) -> int:
-        return self.N // self.B
+        return (self.N + self.B - 1) // self.B
 
     def describe(self) -> dict:
         d = asdict(self)
@@ -78,8 +78,10 @@ def paper_configs() -> dict:
 def make_inputs(cfg: SynthConfig):
     """Returns (Q [L,N,Hq,d], K [L,N,Hkv,d], V [L,N,Hkv,d]) as contiguous bf16 CPU tensors."""
     L, N, Hq, Hkv, d, B = cfg.L, cfg.N, cfg.Hq, cfg.Hkv, cfg.d, cfg.B
-    assert N % B == 0 and Hq % Hkv == 0
-    M, G = N // B, Hq // Hkv
+    assert Hq % Hkv == 0
+    n_keep = N                       # a length that is not a multiple of B is generated padded, then cut
+    M, G = (N + B - 1) // B, Hq // Hkv
+    N = M * B
     g = torch.Generator(device="cpu")
     g.manual_seed(cfg.seed)
 
@@ -123,6 +125,8 @@ def make_inputs(cfg: SynthConfig):
             k[bb, pos[bb, hh], hh] = cfg.nu * math.sqrt(d) * u
         K[l] = k.view(N, Hkv, d).to(torch.bfloat16)
         del k
+    if n_keep != N:
+        Q, K, V = (t[:, :n_keep].contiguous() for t in (Q, K, V))
     return Q, K, V
 
 

@@ -52,7 +52,6 @@ def test_shape_checks_reject_before_launch(lib):
         (RbsShape(1, 1024, 4, 2, 64, 128), UNSUPPORTED),    # head_dim
         (RbsShape(1, 1024, 4, 2, 128, 32), UNSUPPORTED),    # block size
         (RbsShape(1, 1024, 4, 2, 128, 512), UNSUPPORTED),
-        (RbsShape(1, 1000, 4, 2, 128, 128), UNSUPPORTED),   # ragged length
         (RbsShape(1, 1024, 3, 2, 128, 128), UNSUPPORTED),   # heads not divisible
         (RbsShape(0, 1024, 4, 2, 128, 128), INVALID),
     ]

@@ -58,6 +58,10 @@ CASES = {
                             n_sink=2, n_local=3, n_recent=2),
     "gqa_b256": SynthConfig("gqa_b256", N=256 * 37, Hq=4, Hkv=2, B=256, sigma=(0.1, 1.0), seed=34, n_sink=1, n_local=2,
                             n_recent=1),
+    # sequence lengths that are not a multiple of the block: short last key / query block
+    "ragged_n_b128": SynthConfig("ragged_n_b128", N=128 * 21 + 37, Hq=4, Hkv=2, B=128, sigma=(0.1, 1.0), seed=35),
+    "ragged_n_b64": SynthConfig("ragged_n_b64", N=64 * 45 + 63, Hq=2, Hkv=1, B=64, sigma=0.5, seed=36),
+    "ragged_n_b256": SynthConfig("ragged_n_b256", N=256 * 9 + 100, Hq=2, Hkv=2, B=256, sigma=0.5, seed=37),
     "lognormal_b128": SynthConfig("lognormal_b128", N=128 * 40, Hq=2, Hkv=2, B=128, sigma=0.5, sigma_ln=0.5,
                                   p_needle=0.05, seed=33),
 }
@@ -167,7 +171,7 @@ def test_sparse_attention_parity(case):
                 o_ref, lse_ref = orc.masked_attention_block(case["Q64"][l, :, h], case["K64"][l, :, hk],
                                                             case["V64"][l, :, hk], final[l, h, i], i, B)
                 want.append(o_ref); want_lse.append(lse_ref)
-                got.append(O[l, i * B:(i + 1) * B, h]); got_lse.append(lse[l, h, i * B:(i + 1) * B])
+                got.append(O[l, i * B:min(cfg.N, (i + 1) * B), h]); got_lse.append(lse[l, h, i * B:min(cfg.N, (i + 1) * B)])
             _check_output(np.concatenate(got), np.concatenate(want))
             assert np.allclose(np.concatenate(got_lse), np.concatenate(want_lse), atol=2e-3, rtol=1e-4)
 
@@ -199,7 +203,7 @@ def test_dense_attention_sampled_rows(case):
     got, want = [], []
     for i in (0, 1, M // 3, M - 1):
         o_ref, _ = orc.masked_attention_block(case["Q64"][l, :, h], case["K64"][l, :, h // G], case["V64"][l, :, h // G], full, i, B)
-        want.append(o_ref); got.append(O[l, i * B:(i + 1) * B, h])
+        want.append(o_ref); got.append(O[l, i * B:min(cfg.N, (i + 1) * B), h])
     _check_output(np.concatenate(got), np.concatenate(want))
 
 

@@ -418,3 +418,25 @@ def test_end_to_end_gqa_wrapper_uses_the_right_kv_head():
             one = orc.select_head(Q[l, :, h], c, r, beta, B, 0.22, 0.18, 1, 1, 1)
             assert np.array_equal(ref.selection[l][h].final, one.final)
             assert ref.density[l, h] == one.density
+
+
+def test_short_last_block_selection_is_causal_and_uses_its_own_tokens():
+    # cutting tokens off the end must not change any earlier query block's row (causality), and the short last
+    # query block scores exactly like a direct evaluation of Eq. block_aggregation over its remaining tokens
+    B, d = 8, 16
+    Q, K, _ = _random_head(26, M=12, B=B, d=d)
+    cut = 5
+    Qs, Ks = Q[:-cut], K[:-cut]
+    c, r = orc.block_stats(K, B)
+    cs, rs = orc.block_stats(Ks, B)
+    assert np.array_equal(c[:-1], cs[:-1]) and np.array_equal(r[:-1], rs[:-1])
+    beta = np.linspace(0, 1, 12)                    # same beta on both sides: the quantiles see the changed last radius
+    full = orc.select_head(Q, c, r, beta, B, 0.22, 0.18, 1, 1, 0)
+    short = orc.select_head(Qs, cs, rs, beta, B, 0.22, 0.18, 1, 1, 0)
+    assert np.array_equal(full.final[:-1, :-1], short.final[:-1, :-1])
+    i = 11
+    lb, lr = orc.branch_logits(Qs[i * B:], cs, rs, beta)
+    Sb = np.exp(lb / math.sqrt(d)).sum(0)
+    Sr = np.exp(lr / math.sqrt(d)).sum(0)
+    want = (Sb >= 0.22 * Sb.max()) | (Sr >= 0.18 * Sr.max()) | orc.forced_blocks(i, 12, 1, 1, 0)
+    assert np.array_equal(short.final[i], want)
