@@ -127,6 +127,29 @@ RBS_API rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, rbs_
                               void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The same two steps for a range of query blocks only (chunked prefill; prefill against a key/value prefix).
+ * Algorithm 1 treats every query block independently (its third loop and the sparse attention), so a caller may
+ * process the queries of tokens [q_start_block * B, q_start_block * B + n_q_tokens) in one call and the rest in
+ * others, against the keys / values / statistics of the whole sequence (`shape->seqlen` tokens; keys after a query
+ * are hidden by causality, so they need not be final yet).  In these calls
+ *   - Q, O hold only the chunk's tokens (token 0 of the tensor = first token of the chunk), lse is [L][Hq][n_q_tokens];
+ *   - mask / debug masks are [L][Hq][Mq][W] with Mq = ceil(n_q_tokens / B) rows (row 0 = query block q_start_block)
+ *     and W = ceil(M / 32) words per row as usual;
+ *   - density[l][h] = kept pairs of the chunk / causal pairs of the chunk (sum over its query blocks i of i + 1);
+ *   - the "recent" rule still refers to the last n_recent query blocks of the whole sequence.
+ * The chunk must start on a block boundary, lie inside the sequence, and may end inside a block only at the end of
+ * the sequence (RBS_ERR_INVALID_ARG otherwise).  rbs_select_chunk recomputes stats.beta / stats.rq from all M radii on
+ * every call.  With q_start_block = 0 and n_q_tokens = seqlen they are rbs_select / rbs_sparse_prefill.
+ */
+RBS_API rbs_status rbs_select_chunk(const rbs_shape* shape, int q_start_block, int n_q_tokens, rbs_tensor Q,
+                                    rbs_stats stats, float alpha_base, float alpha_rescue, int n_sink, int n_local,
+                                    int n_recent, uint32_t* mask, float* density, uint32_t* dbg_base_mask,
+                                    uint32_t* dbg_rescue_mask, void* workspace, size_t workspace_bytes, void* stream);
+RBS_API rbs_status rbs_sparse_prefill_chunk(const rbs_shape* shape, int q_start_block, int n_q_tokens, rbs_tensor Q,
+                                            rbs_tensor K, rbs_tensor V, const uint32_t* mask, rbs_tensor O, float* lse,
+                                            float softmax_scale, void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * The selector variants the paper compares with in a shared backend (Sec. 4.2, the selector ablation), through
  * the same kernels:
  *   RBS_SELECTOR_RBS            the method itself; identical to rbs_select.

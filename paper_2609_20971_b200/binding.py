@@ -57,6 +57,11 @@ def load_library() -> ctypes.CDLL:
     lib.rbs_block_stats.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, vp]
     lib.rbs_select.restype = i
     lib.rbs_select.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, f, f, i, i, i, vp, vp, vp, vp, vp, sz, vp]
+    lib.rbs_select_chunk.restype = i
+    lib.rbs_select_chunk.argtypes = [ctypes.POINTER(RbsShape), i, i, RbsTensor, RbsStats, f, f, i, i, i, vp, vp, vp, vp, vp, sz, vp]
+    lib.rbs_sparse_prefill_chunk.restype = i
+    lib.rbs_sparse_prefill_chunk.argtypes = [ctypes.POINTER(RbsShape), i, i, RbsTensor, RbsTensor, RbsTensor, vp, RbsTensor,
+                                             vp, f, vp, sz, vp]
     lib.rbs_select_variant.restype = i
     lib.rbs_select_variant.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, i, f, f, i, i, i, vp, vp, vp, vp, vp, sz, vp]
     lib.rbs_select_static.restype = i
@@ -216,4 +221,42 @@ def rbs_sparse_prefill(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, mask: 
     _check(lib.rbs_sparse_prefill(ctypes.byref(shape), _tensor(Q), _tensor(K), _tensor(V), _ptr(mask), _tensor(out),
                                   _ptr(lse), softmax_scale, _ptr(workspace),
                                   0 if workspace is None else workspace.numel(), _stream()), "rbs_sparse_prefill")
+    return (out, lse) if return_lse else out
+
+
+def rbs_select_chunk(Q: torch.Tensor, stats: BlockStats, block: int, seqlen: int, q_start_block: int,
+                     alpha_base: float = 0.22, alpha_rescue: float = 0.18, n_sink: int = 1, n_local: int = 1,
+                     n_recent: int = 1, *, mask: torch.Tensor | None = None, density: torch.Tensor | None = None,
+                     workspace: torch.Tensor | None = None):
+    """Selection for the query chunk Q [L, Nq, Hq, d] that starts at block `q_start_block` of a sequence of `seqlen`
+    tokens whose statistics are in `stats`.  Returns (mask [L,Hq,Mq,W], density [L,Hq]) of the chunk."""
+    lib = load_library()
+    L, Nq, Hq, d = Q.shape
+    shape = RbsShape(L, seqlen, Hq, stats.centroid.shape[1], d, block)
+    M, Mq = (seqlen + block - 1) // block, (Nq + block - 1) // block
+    if mask is None:
+        mask = torch.empty(L, Hq, Mq, (M + 31) // 32, dtype=torch.int32, device=Q.device)
+    if density is None:
+        density = torch.empty(L, Hq, dtype=torch.float32, device=Q.device)
+    if workspace is None:
+        workspace = torch.empty(max(256, workspace_bytes(RBS_OP_SELECT, shape)), dtype=torch.uint8, device=Q.device)
+    _check(lib.rbs_select_chunk(ctypes.byref(shape), q_start_block, Nq, _tensor(Q), stats.c_struct(), alpha_base,
+                                alpha_rescue, n_sink, n_local, n_recent, _ptr(mask), _ptr(density), None, None,
+                                _ptr(workspace), workspace.numel(), _stream()), "rbs_select_chunk")
+    return mask, density
+
+
+def rbs_sparse_prefill_chunk(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, mask: torch.Tensor | None, block: int,
+                             q_start_block: int, *, out: torch.Tensor | None = None, return_lse: bool = False,
+                             softmax_scale: float = 0.0):
+    """Attention for the query chunk Q [L, Nq, Hq, d] starting at block `q_start_block`, against K, V [L, N, Hkv, d]."""
+    lib = load_library()
+    L, Nq, Hq, d = Q.shape
+    shape = RbsShape(L, K.shape[1], Hq, K.shape[2], d, block)
+    if out is None:
+        out = torch.empty_like(Q)
+    lse = torch.empty(L, Hq, Nq, dtype=torch.float32, device=Q.device) if return_lse else None
+    _check(lib.rbs_sparse_prefill_chunk(ctypes.byref(shape), q_start_block, Nq, _tensor(Q), _tensor(K), _tensor(V),
+                                        _ptr(mask), _tensor(out), _ptr(lse), softmax_scale, None, 0, _stream()),
+           "rbs_sparse_prefill_chunk")
     return (out, lse) if return_lse else out

@@ -22,6 +22,14 @@ rbs_status check_tensor(const rbs_tensor& t) {
   return RBS_OK;
 }
 
+rbs_status check_chunk(const Dims& x, int q_start_block, int n_q_tokens) {
+  if (q_start_block < 0 || n_q_tokens <= 0) return RBS_ERR_INVALID_ARG;
+  const long long end = static_cast<long long>(q_start_block) * x.B + n_q_tokens;
+  if (end > x.N) return RBS_ERR_INVALID_ARG;
+  if (n_q_tokens % x.B != 0 && end != x.N) return RBS_ERR_INVALID_ARG;
+  return RBS_OK;
+}
+
 SelectWorkspace select_workspace(const Dims& x) {
   SelectWorkspace w;
   w.Mpad = (x.M + 127) / 128 * 128;

@@ -31,6 +31,10 @@ inline Dims make_dims(const rbs_shape& s) {
 // Host-side argument checks shared by the entry points.
 rbs_status check_shape(const rbs_shape* shape);
 rbs_status check_tensor(const rbs_tensor& t);
+struct Dims;
+// A query chunk must start on a block boundary, lie inside the sequence, and may end inside a block only at the
+// end of the sequence.
+rbs_status check_chunk(const Dims& x, int q_start_block, int n_q_tokens);
 
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 

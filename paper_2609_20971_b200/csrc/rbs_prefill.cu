@@ -15,6 +15,7 @@ struct PrefillParams {
   float* lse;            // nullable
   int M, W, L, Hq, G, N;
   int R;   // 128-row tiles per block (tensor-core path): block / 128
+  int q0, Mq, Nq;   // this call's queries: first query block (global index), number of blocks, number of tokens
   float scale_log2;
 };
 
@@ -60,15 +61,16 @@ prefill_mma_kernel(const PrefillParams p) {
   const int gq = lane >> 2, tq = lane & 3;
 
   const int per_i = p.L * p.Hq;
-  const int i = p.M - 1 - static_cast<int>(blockIdx.x / per_i);
+  const int il = p.Mq - 1 - static_cast<int>(blockIdx.x / per_i);   // query block inside this call's chunk
+  const int i = p.q0 + il;                                            // its position in the sequence
   const int rem = static_cast<int>(blockIdx.x % per_i);
   const int l = rem / p.Hq, h = rem % p.Hq, hk = h / p.G;
-  const uint32_t* mrow = p.mask ? p.mask + ((static_cast<int64_t>(l) * p.Hq + h) * p.M + i) * p.W : nullptr;
+  const uint32_t* mrow = p.mask ? p.mask + ((static_cast<int64_t>(l) * p.Hq + h) * p.Mq + il) * p.W : nullptr;
 
-  const __nv_bfloat16* qbase = p.Q + l * p.qsb + static_cast<int64_t>(i) * B * p.qst + h * p.qsh;
+  const __nv_bfloat16* qbase = p.Q + l * p.qsb + static_cast<int64_t>(il) * B * p.qst + h * p.qsh;
   const __nv_bfloat16* kbase = p.K + l * p.ksb + hk * p.ksh;
   const __nv_bfloat16* vbase = p.V + l * p.vsb + hk * p.vsh;
-  __nv_bfloat16* obase = p.O + l * p.osb + static_cast<int64_t>(i) * B * p.ost + h * p.osh;
+  __nv_bfloat16* obase = p.O + l * p.osb + static_cast<int64_t>(il) * B * p.ost + h * p.osh;
 
   auto load_kv = [&](int b, int stage) {
     const __nv_bfloat16* ks = kbase + static_cast<int64_t>(b) * B * p.kst;
@@ -85,13 +87,13 @@ prefill_mma_kernel(const PrefillParams p) {
 
   int b_cur = next_block(mrow, -1, i);
   const int row0 = warp * 16 + gq;  // this thread's first query row inside the block (second: +8)
-  const int q_rows = min(B, p.N - i * B);   // a short last query block: rows past the sequence end are not written
+  const int q_rows = min(B, p.Nq - il * B);   // a short last query block: rows past the sequence end are not written
   if (b_cur < 0) {                  // nothing retained: zero rows, lse = -inf
     for (int c = tid; c < B * 16; c += NTHREADS) {
       const int row = c >> 4, chunk = c & 15;
       if (row < q_rows) *reinterpret_cast<uint4*>(obase + static_cast<int64_t>(row) * p.ost + chunk * 8) = make_uint4(0, 0, 0, 0);
     }
-    if (p.lse && tid < q_rows) p.lse[(static_cast<int64_t>(l) * p.Hq + h) * p.N + i * B + tid] = -INFINITY;
+    if (p.lse && tid < q_rows) p.lse[(static_cast<int64_t>(l) * p.Hq + h) * p.Nq + il * B + tid] = -INFINITY;
     return;
   }
 
@@ -223,7 +225,7 @@ prefill_mma_kernel(const PrefillParams p) {
     if (row0 + 8 < q_rows) *reinterpret_cast<uint32_t*>(o1 + n * 8 + tq * 2) = pack_bf16(acc_o[n][2] * inv1, acc_o[n][3] * inv1);
   }
   if (p.lse && tq == 0) {
-    float* dst = p.lse + (static_cast<int64_t>(l) * p.Hq + h) * p.N + i * B;
+    float* dst = p.lse + (static_cast<int64_t>(l) * p.Hq + h) * p.Nq + il * B;
     if (row0 < q_rows) dst[row0] = (m_run[0] + fast_log2(l_run[0])) * 0.6931471805599453f;
     if (row0 + 8 < q_rows) dst[row0 + 8] = (m_run[1] + fast_log2(l_run[1])) * 0.6931471805599453f;
   }
@@ -267,15 +269,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   // together.  All tiles in flight then read the K/V of one KV head (64 MiB at 128K tokens), which stays in L2;
   // with all KV heads interleaved the K/V tiles of a 128K layer (256 MiB) were re-read from DRAM many times.
   const int R = p.R;
-  const int per_kv = p.M * R * p.G;
+  const int per_kv = p.Mq * R * p.G;
   const int kvid = static_cast<int>(blockIdx.x / per_kv), rem = static_cast<int>(blockIdx.x % per_kv);
   const int Hkv = p.Hq / p.G;
   const int l = kvid / Hkv, hk = kvid % Hkv;
-  const int T = p.M * R - 1 - rem / p.G;   // 128-row query tile
-  const int i = T / R;                      // its query block (mask row)
+  const int Tl = p.Mq * R - 1 - rem / p.G;  // 128-row query tile inside this call's chunk
+  const int T = p.q0 * R + Tl;              // its position in the sequence (in 128-token units)
+  const int i = T / R;                      // its query block
   const int h = hk * p.G + rem % p.G;
-  if (T * 128 >= p.N) return;               // a tile wholly past the sequence end (short last block of 256)
-  const uint32_t* mrow = p.mask ? p.mask + ((static_cast<int64_t>(l) * p.Hq + h) * p.M + i) * p.W : nullptr;
+  if (Tl * 128 >= p.Nq) return;             // a tile wholly past the end of the queries (short last block of 256)
+  const uint32_t* mrow = p.mask ? p.mask + ((static_cast<int64_t>(l) * p.Hq + h) * p.Mq + (i - p.q0)) * p.W : nullptr;
 
   if (tid == 0) {
     mbar_init(smem_u32(&bar_q), 1);
@@ -303,8 +306,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       int b = next_kb(mrow, -1, i, R, T);
       if (b >= 0) {
         mbar_arrive_expect_tx(smem_u32(&bar_q), kTile);
-        tma_load_4d(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, T * B, l);
-        tma_load_4d(smem_u32(sQ + kPanel), &tmQ, smem_u32(&bar_q), 64, h, T * B, l);
+        tma_load_4d(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, Tl * B, l);
+        tma_load_4d(smem_u32(sQ + kPanel), &tmQ, smem_u32(&bar_q), 64, h, Tl * B, l);
       }
       for (int j = 0; b >= 0; ++j, b = next_kb(mrow, b, i, R, T)) {
         if (j > 0 && !mbar_wait(smem_u32(&bar_s), (j - 1) & 1, status, kWaitStageFree)) break;   // S_{j-1} done: K free
@@ -457,9 +460,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       l_sum += (a0 + a1) + (a2 + a3);
     }
     // epilogue: O / l -> bf16 -> global
-    __nv_bfloat16* orow = p.O + l * p.osb + (static_cast<int64_t>(T) * B + row) * p.ost + h * p.osh;
-    float* lse_dst = p.lse ? p.lse + (static_cast<int64_t>(l) * p.Hq + h) * p.N + T * B + row : nullptr;
-    const bool in_seq = T * B + row < p.N;   // rows of a short last block past the sequence end are not written
+    __nv_bfloat16* orow = p.O + l * p.osb + (static_cast<int64_t>(Tl) * B + row) * p.ost + h * p.osh;
+    float* lse_dst = p.lse ? p.lse + (static_cast<int64_t>(l) * p.Hq + h) * p.Nq + Tl * B + row : nullptr;
+    const bool in_seq = Tl * B + row < p.Nq;   // rows of a short last block past the sequence end are not written
     if (!any_block) {
       if (in_seq) {
 #pragma unroll
@@ -497,14 +500,14 @@ static rbs_status launch_prefill_tc(const PrefillParams& p, const rbs_tensor& Q,
                                     const rbs_tensor& V, int Hkv, cudaStream_t s) {
   CUtensorMap tmQ, tmK, tmV;
   rbs_status st;
-  if ((st = make_tmap_lthd(&tmQ, Q.ptr, p.L, p.N, p.Hq, kHeadDim, Q.stride_batch, Q.stride_token, Q.stride_head, 64, 128, true)) != RBS_OK) return st;
+  if ((st = make_tmap_lthd(&tmQ, Q.ptr, p.L, p.Nq, p.Hq, kHeadDim, Q.stride_batch, Q.stride_token, Q.stride_head, 64, 128, true)) != RBS_OK) return st;
   if ((st = make_tmap_lthd(&tmK, K.ptr, p.L, p.N, Hkv, kHeadDim, K.stride_batch, K.stride_token, K.stride_head, 64, 128, true)) != RBS_OK) return st;
   if ((st = make_tmap_lthd(&tmV, V.ptr, p.L, p.N, Hkv, kHeadDim, V.stride_batch, V.stride_token, V.stride_head, 64, 128, true)) != RBS_OK) return st;
   unsigned int* status = device_status_ptr();
   if (status == nullptr) return RBS_ERR_CUDA;
   const size_t smem = 3 * 2 * 128 * 128;
   RBS_CUDA_OK(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-  const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.M * p.R;
+  const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.Mq * p.R;
   if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
   prefill_tc_kernel<<<static_cast<unsigned>(n_cta), kPfThreads, smem, s>>>(tmQ, tmK, tmV, p, status);
   RBS_CUDA_OK(cudaGetLastError());
@@ -515,7 +518,7 @@ template <int B>
 static rbs_status launch_prefill(const PrefillParams& p, cudaStream_t s) {
   const size_t smem = static_cast<size_t>(5) * B * 256;
   RBS_CUDA_OK(cudaFuncSetAttribute(prefill_mma_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-  const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.M;
+  const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.Mq;
   if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
   prefill_mma_kernel<B><<<static_cast<unsigned>(n_cta), B * 2, smem, s>>>(p);
   RBS_CUDA_OK(cudaGetLastError());
@@ -524,9 +527,9 @@ static rbs_status launch_prefill(const PrefillParams& p, cudaStream_t s) {
 
 }  // namespace rbs
 
-extern "C" rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, rbs_tensor K, rbs_tensor V,
-                                         const uint32_t* mask, rbs_tensor O, float* lse, float softmax_scale,
-                                         void* workspace, size_t workspace_bytes, void* stream) {
+static rbs_status prefill_impl(const rbs_shape* shape, int q_start_block, int n_q_tokens, rbs_tensor Q, rbs_tensor K,
+                               rbs_tensor V, const uint32_t* mask, rbs_tensor O, float* lse, float softmax_scale,
+                               void* workspace, size_t workspace_bytes, void* stream) {
   using namespace rbs;
   (void)workspace; (void)workspace_bytes;
   rbs_status st = check_shape(shape);
@@ -536,7 +539,10 @@ extern "C" rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, r
     return st;
   if (softmax_scale < 0.f) return RBS_ERR_INVALID_ARG;
   Dims x = make_dims(*shape);
+  if (n_q_tokens < 0) { q_start_block = 0; n_q_tokens = x.N; }
+  if ((st = check_chunk(x, q_start_block, n_q_tokens)) != RBS_OK) return st;
   PrefillParams p;
+  p.q0 = q_start_block; p.Nq = n_q_tokens; p.Mq = (n_q_tokens + x.B - 1) / x.B;
   p.Q = static_cast<const __nv_bfloat16*>(Q.ptr); p.qsb = Q.stride_batch; p.qst = Q.stride_token; p.qsh = Q.stride_head;
   p.K = static_cast<const __nv_bfloat16*>(K.ptr); p.ksb = K.stride_batch; p.kst = K.stride_token; p.ksh = K.stride_head;
   p.V = static_cast<const __nv_bfloat16*>(V.ptr); p.vsb = V.stride_batch; p.vst = V.stride_token; p.vsh = V.stride_head;
@@ -549,4 +555,19 @@ extern "C" rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, r
   p.R = x.B / 128;
   if (x.B >= 128) return launch_prefill_tc(p, Q, K, V, x.Hkv, s);   // tensor-core path (blocks of 128 or 256)
   return launch_prefill<64>(p, s);                                    // blocks of 64: register-softmax mma.sync path
+}
+
+extern "C" rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, rbs_tensor K, rbs_tensor V,
+                                         const uint32_t* mask, rbs_tensor O, float* lse, float softmax_scale,
+                                         void* workspace, size_t workspace_bytes, void* stream) {
+  return prefill_impl(shape, -1, -1, Q, K, V, mask, O, lse, softmax_scale, workspace, workspace_bytes, stream);
+}
+
+extern "C" rbs_status rbs_sparse_prefill_chunk(const rbs_shape* shape, int q_start_block, int n_q_tokens, rbs_tensor Q,
+                                               rbs_tensor K, rbs_tensor V, const uint32_t* mask, rbs_tensor O, float* lse,
+                                               float softmax_scale, void* workspace, size_t workspace_bytes,
+                                               void* stream) {
+  if (n_q_tokens <= 0) return RBS_ERR_INVALID_ARG;
+  return prefill_impl(shape, q_start_block, n_q_tokens, Q, K, V, mask, O, lse, softmax_scale, workspace,
+                      workspace_bytes, stream);
 }

@@ -113,6 +113,7 @@ struct SelectParams {
   const __nv_bfloat16* Q; int64_t qsb, qst, qsh;
   const __nv_bfloat16* chi; const __nv_bfloat16* clo; const float* g; const float* cnorm;
   int M, Mpad, W, L, Hq, G, N;
+  int q0, Mq, Nq;   // this call's queries: first query block (global index), number of blocks, number of tokens
   float scale_log2, t_base, t_rescue;  // thresholds as log2(alpha)
   int n_sink, n_local, n_recent;
   uint32_t* mask; uint32_t* dbg_base; uint32_t* dbg_rescue;
@@ -140,7 +141,8 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int per_i = p.L * p.Hq;
-  const int i = p.M - 1 - static_cast<int>(blockIdx.x / per_i);
+  const int il = p.Mq - 1 - static_cast<int>(blockIdx.x / per_i);   // query block inside this call's chunk
+  const int i = p.q0 + il;                                            // its position in the sequence
   const int rem = static_cast<int>(blockIdx.x % per_i);
   const int l = rem / p.Hq, h = rem % p.Hq, hk = h / p.G;
   const int Hkv = p.Hq / p.G;
@@ -165,8 +167,8 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     if (lane == 0) {
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmChi); tma_prefetch_desc(&tmClo);
       mbar_arrive_expect_tx(smem_u32(&bar_q), 2 * kPanelQ);
-      tma_load_4d(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, i * B, l);
-      tma_load_4d(smem_u32(sQ + kPanelQ), &tmQ, smem_u32(&bar_q), 64, h, i * B, l);
+      tma_load_4d(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, il * B, l);
+      tma_load_4d(smem_u32(sQ + kPanelQ), &tmQ, smem_u32(&bar_q), 64, h, il * B, l);
       // the hi and lo halves of a centroid tile are separate pipeline slots: the hi half of the next tile is
       // fetched as soon as this tile's hi MMAs are done, i.e. under its lo MMAs and its epilogue
       const uint32_t dst = smem_u32(sC);
@@ -233,7 +235,7 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) qn_max = fmaxf(qn_max, __shfl_xor_sync(0xffffffffu, qn_max, o));
     const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
-    const int n_tok = min(B, p.N - i * B);
+    const int n_tok = min(B, p.Nq - il * B);
     for (int bt = 0; ok && bt < n_tiles; ++bt) {
       const int buf = bt & 1;
       ok = mbar_wait(smem_u32(&bar_tfull[buf]), (bt >> 1) & 1, status, kWaitMmaDone);
@@ -337,7 +339,7 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 #pragma unroll
   for (int w = 1; w < kTcThreads / 32; ++w) { mxb = fmaxf(mxb, sRed[w]); mxr = fmaxf(mxr, sRed[16 + w]); }
   const float thr_b = mxb + p.t_base, thr_r = mxr + p.t_rescue;
-  const int64_t mrow = ((static_cast<int64_t>(l) * p.Hq + h) * p.M + i) * p.W;
+  const int64_t mrow = ((static_cast<int64_t>(l) * p.Hq + h) * p.Mq + il) * p.W;
   const bool all_forced = i >= p.M - p.n_recent;
   unsigned int cnt = 0;
   for (int w = warp; w < p.W; w += kTcThreads / 32) {
@@ -362,18 +364,19 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (lane == 0 && cnt) atomicAdd(p.counts + l * p.Hq + h, cnt);
 }
 
-__global__ void density_kernel(const unsigned int* __restrict__ counts, int n, int M, float* __restrict__ density) {
+__global__ void density_kernel(const unsigned int* __restrict__ counts, int n, int q0, int Mq, float* __restrict__ density) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t < n) {
-    const double pairs = 0.5 * static_cast<double>(M) * static_cast<double>(M + 1);
+    // causal pairs of query blocks q0 .. q0 + Mq - 1: sum of (i + 1)
+    const double pairs = static_cast<double>(Mq) * static_cast<double>(q0) + 0.5 * static_cast<double>(Mq) * static_cast<double>(Mq + 1);
     density[t] = static_cast<float>(static_cast<double>(counts[t]) / pairs);
   }
 }
 
 template <int B>
-static rbs_status launch_select_tc(const SelectParams& p, const rbs_tensor& Q, int N, cudaStream_t s) {
+static rbs_status launch_select_tc(const SelectParams& p, const rbs_tensor& Q, cudaStream_t s) {
   CUtensorMap tmQ, tmChi, tmClo;
-  rbs_status st = make_tmap_lthd(&tmQ, Q.ptr, p.L, N, p.Hq, kHeadDim, Q.stride_batch, Q.stride_token, Q.stride_head, 64, B, true);
+  rbs_status st = make_tmap_lthd(&tmQ, Q.ptr, p.L, p.Nq, p.Hq, kHeadDim, Q.stride_batch, Q.stride_token, Q.stride_head, 64, B, true);
   if (st != RBS_OK) return st;
   const int64_t rows = static_cast<int64_t>(p.L) * (p.Hq / p.G) * p.Mpad;
   if ((st = make_tmap_2d(&tmChi, p.chi, rows, kHeadDim, 64, 128)) != RBS_OK) return st;
@@ -385,7 +388,7 @@ static rbs_status launch_select_tc(const SelectParams& p, const rbs_tensor& Q, i
                       (B + 32) * sizeof(float) + 2 * static_cast<size_t>(n_tiles_max) * 128 * sizeof(float);
   auto kern = select_tc_kernel<B>;
   RBS_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-  const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.M;
+  const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.Mq;
   if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
   kern<<<static_cast<unsigned>(n_cta), kTcThreads, smem, s>>>(tmQ, tmChi, tmClo, p, status);
   RBS_CUDA_OK(cudaGetLastError());
@@ -394,7 +397,9 @@ static rbs_status launch_select_tc(const SelectParams& p, const rbs_tensor& Q, i
 
 }  // namespace rbs
 
-static rbs_status select_impl(const rbs_shape* shape, rbs_tensor Q, rbs_stats stats, int beta_mode, float alpha_base,
+// q_start_block / n_q_tokens: the queries of this call are tokens [q_start_block * B, q_start_block * B + n_q_tokens)
+// of the sequence; Q, mask and density cover only them (n_q_tokens < 0: the whole sequence).
+static rbs_status select_impl(const rbs_shape* shape, int q_start_block, int n_q_tokens, rbs_tensor Q, rbs_stats stats, int beta_mode, float alpha_base,
                               float alpha_rescue, int n_sink, int n_local, int n_recent, uint32_t* mask,
                               float* density, uint32_t* dbg_base_mask, uint32_t* dbg_rescue_mask,
                               void* workspace, size_t workspace_bytes, void* stream) {
@@ -407,6 +412,8 @@ static rbs_status select_impl(const rbs_shape* shape, rbs_tensor Q, rbs_stats st
   if (!(alpha_base > 0.f) || !(alpha_rescue > 0.f)) return RBS_ERR_INVALID_ARG;
   if (n_sink < 0 || n_local < 0 || n_recent < 0) return RBS_ERR_INVALID_ARG;
   Dims x = make_dims(*shape);
+  if (n_q_tokens < 0) { q_start_block = 0; n_q_tokens = x.N; }
+  if ((st = check_chunk(x, q_start_block, n_q_tokens)) != RBS_OK) return st;
   SelectWorkspace ws = select_workspace(x);
   if (workspace == nullptr || workspace_bytes < ws.bytes) return RBS_ERR_WORKSPACE;
   if (reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return RBS_ERR_WORKSPACE;
@@ -436,14 +443,15 @@ static rbs_status select_impl(const rbs_shape* shape, rbs_tensor Q, rbs_stats st
   p.Q = static_cast<const __nv_bfloat16*>(Q.ptr); p.qsb = Q.stride_batch; p.qst = Q.stride_token; p.qsh = Q.stride_head;
   p.chi = chi; p.clo = clo; p.g = g; p.cnorm = cnorm;
   p.M = x.M; p.Mpad = ws.Mpad; p.W = x.W; p.L = x.L; p.Hq = x.Hq; p.G = x.G; p.N = x.N;
+  p.q0 = q_start_block; p.Nq = n_q_tokens; p.Mq = (n_q_tokens + x.B - 1) / x.B;
   p.scale_log2 = scale_log2; p.t_base = log2f(alpha_base); p.t_rescue = log2f(alpha_rescue);
   p.n_sink = n_sink; p.n_local = n_local; p.n_recent = n_recent;
   p.mask = mask; p.dbg_base = dbg_base_mask; p.dbg_rescue = dbg_rescue_mask; p.counts = counts;
-  if (x.B == 256) st = launch_select_tc<256>(p, Q, x.N, s);
-  else st = (x.B == 128) ? launch_select_tc<128>(p, Q, x.N, s) : launch_select_tc<64>(p, Q, x.N, s);
+  if (x.B == 256) st = launch_select_tc<256>(p, Q, s);
+  else st = (x.B == 128) ? launch_select_tc<128>(p, Q, s) : launch_select_tc<64>(p, Q, s);
   if (st != RBS_OK) return st;
   const int nh = x.L * x.Hq;
-  density_kernel<<<(nh + 127) / 128, 128, 0, s>>>(counts, nh, x.M, density);
+  density_kernel<<<(nh + 127) / 128, 128, 0, s>>>(counts, nh, p.q0, p.Mq, density);
   RBS_CUDA_OK(cudaGetLastError());
   return RBS_OK;
 }
@@ -452,8 +460,17 @@ extern "C" rbs_status rbs_select(const rbs_shape* shape, rbs_tensor Q, rbs_stats
                                  float alpha_rescue, int n_sink, int n_local, int n_recent, uint32_t* mask,
                                  float* density, uint32_t* dbg_base_mask, uint32_t* dbg_rescue_mask,
                                  void* workspace, size_t workspace_bytes, void* stream) {
-  return select_impl(shape, Q, stats, 0, alpha_base, alpha_rescue, n_sink, n_local, n_recent, mask, density,
+  return select_impl(shape, -1, -1, Q, stats, 0, alpha_base, alpha_rescue, n_sink, n_local, n_recent, mask, density,
                      dbg_base_mask, dbg_rescue_mask, workspace, workspace_bytes, stream);
+}
+
+extern "C" rbs_status rbs_select_chunk(const rbs_shape* shape, int q_start_block, int n_q_tokens, rbs_tensor Q,
+                                       rbs_stats stats, float alpha_base, float alpha_rescue, int n_sink, int n_local,
+                                       int n_recent, uint32_t* mask, float* density, uint32_t* dbg_base_mask,
+                                       uint32_t* dbg_rescue_mask, void* workspace, size_t workspace_bytes, void* stream) {
+  if (n_q_tokens <= 0) return RBS_ERR_INVALID_ARG;
+  return select_impl(shape, q_start_block, n_q_tokens, Q, stats, 0, alpha_base, alpha_rescue, n_sink, n_local, n_recent,
+                     mask, density, dbg_base_mask, dbg_rescue_mask, workspace, workspace_bytes, stream);
 }
 
 extern "C" rbs_status rbs_select_variant(const rbs_shape* shape, rbs_tensor Q, rbs_stats stats, rbs_selector which,
@@ -464,13 +481,13 @@ extern "C" rbs_status rbs_select_variant(const rbs_shape* shape, rbs_tensor Q, r
   constexpr float kDisabled = 2.0f;   // alpha > 1 empties a branch
   switch (which) {
     case RBS_SELECTOR_RBS:
-      return select_impl(shape, Q, stats, 0, alpha_base, alpha_rescue, n_sink, n_local, n_recent, mask, density,
+      return select_impl(shape, -1, -1, Q, stats, 0, alpha_base, alpha_rescue, n_sink, n_local, n_recent, mask, density,
                          dbg_base_mask, dbg_rescue_mask, workspace, workspace_bytes, stream);
     case RBS_SELECTOR_CENTROID_ONLY:
-      return select_impl(shape, Q, stats, 1, alpha_base, kDisabled, n_sink, n_local, n_recent, mask, density,
+      return select_impl(shape, -1, -1, Q, stats, 1, alpha_base, kDisabled, n_sink, n_local, n_recent, mask, density,
                          dbg_base_mask, dbg_rescue_mask, workspace, workspace_bytes, stream);
     case RBS_SELECTOR_FULL_L2:
-      return select_impl(shape, Q, stats, 2, kDisabled, alpha_rescue, n_sink, n_local, n_recent, mask, density,
+      return select_impl(shape, -1, -1, Q, stats, 2, kDisabled, alpha_rescue, n_sink, n_local, n_recent, mask, density,
                          dbg_base_mask, dbg_rescue_mask, workspace, workspace_bytes, stream);
   }
   return RBS_ERR_INVALID_ARG;

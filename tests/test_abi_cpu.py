@@ -94,3 +94,18 @@ def test_binding_fails_loudly_when_library_is_missing(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(binding.RbsError):
         binding.load_library()
+
+
+def test_chunk_argument_checks(lib):
+    good = RbsShape(1, 1000, 4, 2, 128, 128)          # M = 8, last block short
+    need = lib.rbs_workspace_bytes(1, ctypes.byref(good))
+    p = ctypes.c_void_p(0x1000)
+
+    def sel(q0, nq):
+        return lib.rbs_select_chunk(ctypes.byref(good), q0, nq, _t(), _stats(), 0.22, 0.18, 1, 1, 1, p, p, None, None,
+                                    p, need, None)
+    assert sel(-1, 128) == INVALID and sel(0, 0) == INVALID
+    assert sel(7, 128) == INVALID                      # runs past the end of the sequence
+    assert sel(2, 100) == INVALID                      # ends inside a block that is not the last
+    assert lib.rbs_sparse_prefill_chunk(ctypes.byref(good), 8, 64, _t(), _t(), _t(), None, _t(), None, 0.0, None, 0,
+                                        None) == INVALID

@@ -319,3 +319,29 @@ def test_selector_variants_match_the_oracle_with_fixed_beta():
             s = orc.select_head(Q64[0, :, h], c, r, beta, cfg.B, ab, ar, 1, 1, 1)
             near = (s.margin_base <= MASK_MARGIN) if ab < 1 else (s.margin_rescue <= MASK_MARGIN)
             assert not ((got[0, h] != s.final) & ~near).any()
+
+
+@pytest.mark.parametrize("B,Mtot,cuts", [(128, 23, (0, 7, 16)), (64, 40, (0, 13)), (256, 9, (0, 4))])
+def test_chunked_calls_reproduce_the_whole_sequence(B, Mtot, cuts):
+    """Queries processed in chunks (a KV prefix plus new query blocks) give bit-identical masks and outputs."""
+    from paper_2609_20971_b200 import rbs_select_chunk, rbs_sparse_prefill_chunk
+    cfg = SynthConfig("chunk", N=B * Mtot - 19, Hq=4, Hkv=2, B=B, sigma=(0.1, 1.0), seed=45, n_recent=2)
+    Q, K, V = make_inputs(cfg)
+    Qg, Kg, Vg = Q.cuda(), K.cuda(), V.cuda()
+    stats = rbs_block_stats(Kg, B)
+    mask, dens = rbs_select(Qg, stats, B, 0.22, 0.18, 1, 1, 2)
+    O, lse = rbs_sparse_prefill(Qg, Kg, Vg, mask, B, return_lse=True)
+    Od = rbs_sparse_prefill(Qg, Kg, Vg, None, B)
+    bounds = list(cuts) + [cfg.M]
+    kept = 0.0
+    for q0, q1 in zip(bounds[:-1], bounds[1:]):
+        t0, t1 = q0 * B, min(cfg.N, q1 * B)
+        Qc = Qg[:, t0:t1]                                        # a strided view: no copy
+        mc, dc = rbs_select_chunk(Qc, stats, B, cfg.N, q0, 0.22, 0.18, 1, 1, 2)
+        assert torch.equal(mc, mask[:, :, q0:q1])
+        pairs = sum(i + 1 for i in range(q0, q1))
+        kept += float(dc[0, 0]) * pairs
+        oc, lc = rbs_sparse_prefill_chunk(Qc, Kg, Vg, mc, B, q0, return_lse=True)
+        assert torch.equal(oc, O[:, t0:t1]) and torch.equal(lc, lse[:, :, t0:t1])
+        assert torch.equal(rbs_sparse_prefill_chunk(Qc, Kg, Vg, None, B, q0), Od[:, t0:t1])
+    assert abs(kept / (cfg.M * (cfg.M + 1) / 2) - float(dens[0, 0])) < 1e-6
