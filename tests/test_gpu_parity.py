@@ -345,3 +345,22 @@ def test_chunked_calls_reproduce_the_whole_sequence(B, Mtot, cuts):
         assert torch.equal(oc, O[:, t0:t1]) and torch.equal(lc, lse[:, :, t0:t1])
         assert torch.equal(rbs_sparse_prefill_chunk(Qc, Kg, Vg, None, B, q0), Od[:, t0:t1])
     assert abs(kept / (cfg.M * (cfg.M + 1) / 2) - float(dens[0, 0])) < 1e-6
+
+
+def test_host_pipeline_matches_device_resident_calls():
+    from paper_2609_20971_b200.host import HostPrefill
+    cfg = SynthConfig("host", L=1, N=128 * 37 + 50, Hq=4, Hkv=2, B=128, sigma=(0.1, 1.0), seed=46)
+    Q, K, V = make_inputs(cfg)
+    Qh, Kh, Vh = Q.pin_memory(), K.pin_memory(), V.pin_memory()
+    Oh = torch.empty_like(Qh).pin_memory()
+    hp = HostPrefill(1, cfg.N, cfg.Hq, cfg.Hkv, cfg.d, cfg.B, "cuda:0", chunk_blocks=8)
+    for _ in range(2):                       # second run reuses buffers and streams
+        Oh.zero_()
+        hp.run(Qh, Kh, Vh, Oh)
+        hp.wait()
+        torch.cuda.synchronize()
+        Qg, Kg, Vg = Q.cuda(), K.cuda(), V.cuda()
+        stats = rbs_block_stats(Kg, cfg.B)
+        mask, _ = rbs_select(Qg, stats, cfg.B)
+        O = rbs_sparse_prefill(Qg, Kg, Vg, mask, cfg.B)
+        assert torch.equal(Oh.cuda(), O) and torch.equal(hp.mask(), mask)
