@@ -349,16 +349,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (!ok) break;
         tc_fence_after_sync();
         mma_ts_k64_elect(tmem_o, tmem_s, dv, kIdescPV, 2048 >> 4, j != 0, 0);
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_p1), ph, status, kWaitPReady));         // keys 64..127
+        // K of the next block arrived while the softmax ran; checking it here, before the wait for the second half
+        // of P, keeps that check (about 200 cycles of wait, vote and fence) off the tile's critical path
+        if (b_next >= 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull), ph ^ 1, status, kWaitTmaFull));
+        ok = ok && __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_p1), ph, status, kWaitPReady));   // keys 64..127
         if (!ok) break;
         tc_fence_after_sync();
         mma_ts_k64_elect(tmem_o, tmem_s + 32, dv + static_cast<uint64_t>((4 * 2048) >> 4), kIdescPV, 2048 >> 4, 1, smem_u32(&bar_pv));
-        if (b_next >= 0) {                              // K of the next block arrived while the softmax ran
-          ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull), ph ^ 1, status, kWaitTmaFull));
-          if (!ok) break;
-          tc_fence_after_sync();
-          issue_qk();
-        }
+        if (b_next >= 0) issue_qk();
         b = b_next;
       }
     }
