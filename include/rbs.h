@@ -200,6 +200,22 @@ RBS_API rbs_status rbs_select_static(const rbs_shape* shape, rbs_tensor Q, rbs_s
                                      void* stream);
 
 /*
+ * Group-shared masks under grouped-query attention: replaces, in place, the mask rows of the G query heads that
+ * share a KV head by their union, and recomputes density.  The paper's selector is applied per query head
+ * (Sec. 3.2: the scores S are taken over one head's query block); sharing the union inside a KV group is a
+ * variant with no counterpart in the paper: every head of the group then attends the same key blocks, so a
+ * kernel can fetch each selected K/V block once per group, at the price of a higher density.
+ *   mask    device, [batch][n_q_heads][Mq][W] as written by rbs_select / rbs_select_chunk; updated in place
+ *   density device, [batch][n_q_heads] fp32, overwritten: kept pairs / causal pairs of the call's query blocks
+ *           (the same value for the G heads of a group)
+ *   q_start_block, n_q_tokens: the query range the mask covers, as in rbs_select_chunk (n_q_tokens < 0: the whole
+ *           sequence).
+ * Errors as rbs_select_chunk.  Asynchronous on `stream`; no workspace.
+ */
+RBS_API rbs_status rbs_mask_group_union(const rbs_shape* shape, int q_start_block, int n_q_tokens, uint32_t* mask,
+                                        float* density, void* stream);
+
+/*
  * Kernels that wait on hardware barriers (TMA arrival, tensor-core completion) give every wait an
  * iteration limit.  A wait that runs out records a non-zero code in a device-side status word, lets the
  * kernel drain and return, and leaves the CUDA context usable; outputs of that launch are then

@@ -195,6 +195,16 @@ def density(final: np.ndarray) -> float:
     return float((final & causal).sum()) / float(M * (M + 1) // 2)
 
 
+def group_union(finals) -> np.ndarray:
+    """Group-shared mask under grouped-query attention: a pair is kept for the whole KV group when any of the
+    group's query heads keeps it.  `finals` are the [M, M] masks of the heads of one group.  (A variant: the
+    paper's selector, Sec. 3.2, is per query head and has no such step.)"""
+    out = np.zeros_like(np.asarray(finals[0], dtype=bool))
+    for f in finals:
+        out = out | np.asarray(f, dtype=bool)
+    return out
+
+
 # --------------------------------------------------------------------------------------
 # Sec. 3.3: attention over the retained blocks; Eq. (1): dense causal attention
 # --------------------------------------------------------------------------------------

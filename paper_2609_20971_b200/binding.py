@@ -66,6 +66,8 @@ def load_library() -> ctypes.CDLL:
     lib.rbs_select_variant.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, i, f, f, i, i, i, vp, vp, vp, vp, vp, sz, vp]
     lib.rbs_select_static.restype = i
     lib.rbs_select_static.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, f, f, i, i, i, vp, vp, vp, vp, vp]
+    lib.rbs_mask_group_union.restype = i
+    lib.rbs_mask_group_union.argtypes = [ctypes.POINTER(RbsShape), i, i, vp, vp, vp]
     lib.rbs_sparse_prefill.restype = i
     lib.rbs_sparse_prefill.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsTensor, RbsTensor, vp, RbsTensor,
                                        vp, f, vp, sz, vp]
@@ -202,6 +204,20 @@ def rbs_select_static(Q: torch.Tensor, stats: BlockStats, block: int, alpha_base
     _check(lib.rbs_select_static(ctypes.byref(shape), _tensor(Q), stats.c_struct(), alpha_base, alpha_rescue,
                                  n_sink, n_local, n_recent, _ptr(mask), _ptr(density), _ptr(dbg_base),
                                  _ptr(dbg_rescue), _stream()), "rbs_select_static")
+    return mask, density
+
+
+def rbs_mask_group_union(mask: torch.Tensor, density: torch.Tensor, n_kv_heads: int, block: int, seqlen: int,
+                         q_start_block: int = 0, n_q_tokens: int = -1, head_dim: int = 128):
+    """In place: the mask rows [L,Hq,Mq,W] of the query heads that share a KV head become their union, and
+    `density` [L,Hq] is recomputed (a variant outside the paper's per-head selector)."""
+    lib = load_library()
+    L, Hq = mask.shape[0], mask.shape[1]
+    if not mask.is_contiguous() or mask.dtype != torch.int32 or density.dtype != torch.float32:
+        raise RbsError("mask must be a contiguous int32 tensor [L,Hq,Mq,W] and density fp32 [L,Hq]")
+    shape = RbsShape(L, seqlen, Hq, n_kv_heads, head_dim, block)
+    _check(lib.rbs_mask_group_union(ctypes.byref(shape), q_start_block, n_q_tokens, _ptr(mask), _ptr(density),
+                                    _stream()), "rbs_mask_group_union")
     return mask, density
 
 

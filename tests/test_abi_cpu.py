@@ -109,3 +109,15 @@ def test_chunk_argument_checks(lib):
     assert sel(2, 100) == INVALID                      # ends inside a block that is not the last
     assert lib.rbs_sparse_prefill_chunk(ctypes.byref(good), 8, 64, _t(), _t(), _t(), None, _t(), None, 0.0, None, 0,
                                         None) == INVALID
+
+
+def test_group_union_argument_checks(lib):
+    good = RbsShape(1, 1024, 4, 2, 128, 128)
+    p = ctypes.c_void_p(0x1000)
+    lib.rbs_mask_group_union.argtypes = [ctypes.POINTER(RbsShape), ctypes.c_int, ctypes.c_int, ctypes.c_void_p,
+                                         ctypes.c_void_p, ctypes.c_void_p]
+    assert lib.rbs_mask_group_union(ctypes.byref(good), 0, -1, None, p, None) == INVALID
+    assert lib.rbs_mask_group_union(ctypes.byref(good), 0, -1, p, None, None) == INVALID
+    assert lib.rbs_mask_group_union(ctypes.byref(good), 7, 256, p, p, None) == INVALID      # past the end
+    bad = RbsShape(1, 1024, 3, 2, 128, 128)
+    assert lib.rbs_mask_group_union(ctypes.byref(bad), 0, -1, p, p, None) == UNSUPPORTED

@@ -14,7 +14,7 @@ import pytest
 import torch
 
 from oracle import rbs_oracle as orc
-from paper_2609_20971_b200 import rbs_block_stats, rbs_select, rbs_sparse_prefill
+from paper_2609_20971_b200 import rbs_block_stats, rbs_mask_group_union, rbs_select, rbs_sparse_prefill
 from paper_2609_20971_b200.synth import SynthConfig, make_inputs, paper_configs, to_f64
 
 pytestmark = pytest.mark.gpu
@@ -123,6 +123,27 @@ def test_mask_parity(case):
             assert not np.triu(final[l, h], 1).any()
     pairs = M * (M + 1) // 2
     assert n_mismatch <= max(2, int(2e-3 * pairs * cfg.L * cfg.Hq))   # near-threshold blocks are rare
+
+
+def test_group_union_of_masks(case):
+    """Group-shared variant: bit-exact union of the GPU's own per-head masks inside each KV group, density of it."""
+    cfg = case["cfg"]
+    M, G = cfg.M, cfg.Hq // cfg.Hkv
+    per_head = unpack_mask(case["mask"], M)
+    mask = case["mask"].clone()
+    dens = torch.empty_like(case["density"])
+    rbs_mask_group_union(mask, dens, cfg.Hkv, cfg.B, cfg.N)
+    torch.cuda.synchronize()
+    got = unpack_mask(mask, M)
+    dens = dens.cpu().numpy()
+    for l in range(cfg.L):
+        for hk in range(cfg.Hkv):
+            want = orc.group_union([per_head[l, hk * G + g] for g in range(G)])
+            for g in range(G):
+                assert np.array_equal(got[l, hk * G + g], want)
+                assert abs(dens[l, hk * G + g] - orc.density(want)) <= 1e-6
+    # words past the last block column stay untouched (zero)
+    assert np.array_equal(mask.cpu().numpy()[..., (M + 31) // 32:], case["mask"].cpu().numpy()[..., (M + 31) // 32:])
 
 
 def test_density_parity(case):

@@ -440,3 +440,19 @@ def test_short_last_block_selection_is_causal_and_uses_its_own_tokens():
     Sr = np.exp(lr / math.sqrt(d)).sum(0)
     want = (Sb >= 0.22 * Sb.max()) | (Sr >= 0.18 * Sr.max()) | orc.forced_blocks(i, 12, 1, 1, 0)
     assert np.array_equal(short.final[i], want)
+
+
+def test_group_union_is_a_superset_with_additive_density_bound():
+    """Union over a KV group's heads: contains every head's mask, adds nothing else, density between the
+    largest per-head density and their sum."""
+    rng = np.random.default_rng(5)
+    M = 17
+    causal = np.tril(np.ones((M, M), dtype=bool))
+    heads = [(rng.random((M, M)) < 0.2) & causal for _ in range(4)]
+    u = orc.group_union(heads)
+    for f in heads:
+        assert not (f & ~u).any()
+    assert not (u & ~np.any(np.stack(heads), axis=0)).any()
+    rho = [orc.density(f) for f in heads]
+    assert max(rho) <= orc.density(u) <= sum(rho)
+    assert np.array_equal(orc.group_union([heads[0]]), heads[0])
