@@ -96,3 +96,42 @@ def prefill_host(Qh, Kh, Vh, block: int, device="cuda:0", Oh=None, **select_args
     hp.wait()
     torch.cuda.current_stream(hp.dev).synchronize()
     return Oh, dens
+
+
+def prefill_varlen(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, cu_seqlens, block: int, *, out=None,
+                   alpha_base: float = 0.22, alpha_rescue: float = 0.18, n_sink: int = 1, n_local: int = 1,
+                   n_recent: int = 1, streams=None):
+    """A batch of prompts of different lengths packed along the token axis (no padding, nothing concatenated across
+    prompts: every prompt is selected and attended on its own, as in Sec. 4.1).
+
+    Q [T, Hq, d], K and V [T, Hkv, d] are CUDA bf16 tensors holding the prompts back to back; `cu_seqlens` (host
+    ints, length n + 1, cu_seqlens[0] = 0, cu_seqlens[-1] = T) gives the boundaries.  Each prompt becomes one call of
+    rbs_block_stats / rbs_select / rbs_sparse_prefill on a view of the packed buffers (the library takes strides,
+    so nothing is copied); prompts are spread round-robin over `streams` (default: the current stream only).
+    Returns (O [T, Hq, d], densities: list of [1, Hq] tensors, one per prompt)."""
+    from .binding import rbs_select, rbs_sparse_prefill
+    cu = [int(x) for x in cu_seqlens]
+    if len(cu) < 2 or cu[0] != 0 or cu[-1] != Q.shape[0] or any(b <= a for a, b in zip(cu, cu[1:])):
+        raise ValueError("cu_seqlens must start at 0, end at the number of packed tokens and increase strictly")
+    if out is None:
+        out = torch.empty_like(Q)
+    cur = torch.cuda.current_stream(Q.device)
+    streams = list(streams) if streams else [cur]
+    for s in streams:
+        if s != cur:
+            s.wait_stream(cur)
+    densities = []
+    for k, (t0, t1) in enumerate(zip(cu, cu[1:])):
+        s = streams[k % len(streams)]
+        with torch.cuda.stream(s):
+            q, kk, v, o = (t[t0:t1].unsqueeze(0) for t in (Q, K, V, out))
+            stats = rbs_block_stats(kk, block)
+            mask, dens = rbs_select(q, stats, block, alpha_base, alpha_rescue, n_sink, n_local, n_recent)
+            rbs_sparse_prefill(q, kk, v, mask, block, out=o)
+            densities.append(dens)
+            for t in (stats.centroid, stats.radius, stats.beta, stats.rq, mask, dens):
+                t.record_stream(s)
+    for s in streams:
+        if s != cur:
+            cur.wait_stream(s)
+    return out, densities

@@ -385,3 +385,33 @@ def test_host_pipeline_matches_device_resident_calls():
         mask, _ = rbs_select(Qg, stats, cfg.B)
         O = rbs_sparse_prefill(Qg, Kg, Vg, mask, cfg.B)
         assert torch.equal(Oh.cuda(), O) and torch.equal(hp.mask(), mask)
+
+
+def test_varlen_batch_equals_one_call_per_prompt():
+    """Prompts of different lengths packed back to back: each is selected and attended on its own (Sec. 4.1:
+    requests are not concatenated), so the packed call must reproduce the single-prompt calls bit for bit, and the
+    oracle's attention on sampled rows."""
+    from paper_2609_20971_b200.host import prefill_varlen
+    dev = torch.device("cuda:0")
+    B, Hq, Hkv = 128, 4, 2
+    lens = [128 * 9 + 17, 128 * 3, 100, 128 * 14 + 127]
+    parts = [make_inputs(SynthConfig(f"varlen{k}", N=n, Hq=Hq, Hkv=Hkv, B=B, sigma=0.5, seed=70 + k)) for k, n in enumerate(lens)]
+    Qp, Kp, Vp = (torch.cat([p[j][0] for p in parts], dim=0).to(dev) for j in range(3))
+    cu = np.concatenate([[0], np.cumsum(lens)])
+    streams = [torch.cuda.Stream(dev), torch.cuda.Stream(dev)]
+    O, dens = prefill_varlen(Qp, Kp, Vp, cu, B, streams=streams)
+    torch.cuda.synchronize()
+    for k, (Q, K, V) in enumerate(parts):
+        Qg, Kg, Vg = Q.to(dev), K.to(dev), V.to(dev)
+        stats = rbs_block_stats(Kg, B)
+        mask, d1 = rbs_select(Qg, stats, B)
+        O1 = rbs_sparse_prefill(Qg, Kg, Vg, mask, B)
+        torch.cuda.synchronize()
+        assert torch.equal(O[cu[k]:cu[k + 1]], O1[0])
+        assert torch.equal(dens[k], d1)
+    # oracle check on the shortest prompt (one short block: dense causal attention over 100 tokens)
+    k = 2
+    Q64, K64, V64 = (to_f64(t) for t in parts[k])
+    ref, _ = orc.dense_causal_attention(Q64[0, :, 0], K64[0, :, 0], V64[0, :, 0])
+    got = O[cu[k]:cu[k + 1], 0].float().cpu().numpy()
+    assert np.abs(got - ref).max() <= OUT_MAX_ABS
