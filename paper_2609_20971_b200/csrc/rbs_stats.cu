@@ -7,13 +7,13 @@
 namespace rbs {
 
 // ---------------------------------------------------------------------------------------------
-// Every warp owns one shared-memory slot, fetches its own tiles with TMA
+// Every warp owns NS shared-memory slots used in turn, fetches its own tiles with TMA
 // (two 128-byte-swizzled panels of 64 columns) and reduces them alone, so warps never wait for one
-// another.  Pass 1: lanes own 4 columns and walk the rows (column sums, no cross-lane traffic).
+// another; with NS = 2 the next tile is already on its way while the current one is reduced.  Pass 1: lanes own 4 columns and walk the rows (column sums, no cross-lane traffic).
 // Pass 2: lanes own rows and walk the columns (row distances, no cross-lane traffic); the swizzle
 // keeps both access patterns free of bank conflicts.
 // ---------------------------------------------------------------------------------------------
-template <int B, int NW>
+template <int B, int NW, int NS>
 __global__ void __launch_bounds__(NW * 32, 1)
 block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, int M, int Hkv, int N,
                         float* __restrict__ centroid, float* __restrict__ radius, unsigned int* status) {
@@ -21,20 +21,24 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
   constexpr uint32_t kSlot = 2 * kPanel;
   constexpr int RJ = B / 32;                  // rows per lane in pass 2
   extern __shared__ __align__(1024) unsigned char smem[];
-  __shared__ __align__(8) uint64_t full_bar[NW];
+  __shared__ __align__(8) uint64_t full_bar[NW * NS];
+  // half of the warp's centroid (64 columns) at a time, re-read by every lane in pass 2; the whole of it would not
+  // fit beside the tile slots
+  __shared__ __align__(16) float s_cen[NW][kHeadDim / 2];
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const uint32_t bar = smem_u32(&full_bar[warp]);
-  const uint32_t slot = smem_u32(smem) + warp * kSlot;
+  const uint32_t bar0 = smem_u32(&full_bar[warp * NS]);
+  const uint32_t slot0 = smem_u32(smem) + warp * NS * kSlot;
   if (lane == 0) {
-    mbar_init(bar, 1);
+    for (int k = 0; k < NS; ++k) mbar_init(bar0 + 8 * k, 1);
     mbar_fence_init();
   }
   __syncwarp();
 
   const int stride = gridDim.x * NW;
   int t = warp * gridDim.x + blockIdx.x;
-  auto issue = [&](int tile) {
+  auto issue = [&](int tile, int buf) {
+    const uint32_t bar = bar0 + 8 * buf, slot = slot0 + buf * kSlot;
     int idx = tile;
     const int hk = idx % Hkv; idx /= Hkv;
     const int b = idx % M;
@@ -43,14 +47,19 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
     tma_load_4d(slot, &tmK, bar, 0, hk, b * B, l);
     tma_load_4d(slot + kPanel, &tmK, bar, 64, hk, b * B, l);
   };
-  if (lane == 0 && t < n_tiles) issue(t);
+  if (lane == 0) {
+    for (int k = 0; k < NS; ++k)
+      if (t + k * stride < n_tiles) issue(t + k * stride, k);
+  }
 
   // pass-1 addressing: lane owns 8 bytes (4 columns): 16-byte chunk c16 = lane / 2, half = lane % 2
   const int c16 = lane >> 1, cp = c16 & 7;
-  const uint32_t p1_base = slot + (c16 >> 3) * kPanel + (lane & 1) * 8;
-  uint32_t phase = 0;
-  for (; t < n_tiles; t += stride, phase ^= 1) {
-    if (!mbar_wait(bar, phase, status, kWaitTmaFull)) break;
+  for (int it = 0; t < n_tiles; t += stride, ++it) {
+    const int buf = it % NS;
+    const uint32_t phase = (it / NS) & 1;
+    const uint32_t slot = slot0 + buf * kSlot;
+    const uint32_t p1_base = slot + (c16 >> 3) * kPanel + (lane & 1) * 8;
+    if (!mbar_wait(bar0 + 8 * buf, phase, status, kWaitTmaFull)) break;
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll 4
     for (int r8 = 0; r8 < B; r8 += 8) {
@@ -80,12 +89,14 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
     const int sw = lane & 7;
 #pragma unroll
     for (int c = 0; c < 16; ++c) {
-      // centroid columns 8c..8c+7 live in lanes 2c and 2c+1
-      float4 ca, cb;
-      ca.x = __shfl_sync(0xffffffffu, cen.x, 2 * c); ca.y = __shfl_sync(0xffffffffu, cen.y, 2 * c);
-      ca.z = __shfl_sync(0xffffffffu, cen.z, 2 * c); ca.w = __shfl_sync(0xffffffffu, cen.w, 2 * c);
-      cb.x = __shfl_sync(0xffffffffu, cen.x, 2 * c + 1); cb.y = __shfl_sync(0xffffffffu, cen.y, 2 * c + 1);
-      cb.z = __shfl_sync(0xffffffffu, cen.z, 2 * c + 1); cb.w = __shfl_sync(0xffffffffu, cen.w, 2 * c + 1);
+      if ((c & 7) == 0) {   // columns 64 (c / 8) .. +63 of the centroid live in lanes 16 (c / 8) .. +15
+        __syncwarp();
+        if ((lane >> 4) == (c >> 3)) reinterpret_cast<float4*>(s_cen[warp])[lane & 15] = cen;
+        __syncwarp();
+      }
+      // centroid columns 8c..8c+7: two broadcast reads (all lanes, same address)
+      const float4 ca = reinterpret_cast<const float4*>(s_cen[warp])[2 * (c & 7)];
+      const float4 cb = reinterpret_cast<const float4*>(s_cen[warp])[2 * (c & 7) + 1];
       const uint32_t col = (c >> 3) * kPanel + (((c & 7) ^ sw) << 4);
 #pragma unroll
       for (int j = 0; j < RJ; ++j) {
@@ -108,9 +119,9 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
     for (int j = 0; j < RJ; ++j)
       if (lane + 32 * j < rows_valid) rmax = fmaxf(rmax, q[j]);
     __syncwarp();   // every lane is done reading the slot
-    if (lane == 0 && t + stride < n_tiles) {
+    if (lane == 0 && t + NS * stride < n_tiles) {
       fence_proxy_async_smem();
-      issue(t + stride);
+      issue(t + NS * stride, buf);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, o));
@@ -118,7 +129,7 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
   }
 }
 
-template <int B, int NW>
+template <int B, int NW, int NS>
 static rbs_status launch_stats_warp(const rbs_tensor& K, const Dims& x, const rbs_stats& stats, cudaStream_t s) {
   CUtensorMap tm;
   rbs_status st = make_tmap_lthd(&tm, K.ptr, x.L, x.N, x.Hkv, x.d, K.stride_batch, K.stride_token, K.stride_head,
@@ -126,8 +137,8 @@ static rbs_status launch_stats_warp(const rbs_tensor& K, const Dims& x, const rb
   if (st != RBS_OK) return st;
   unsigned int* status = device_status_ptr();
   if (status == nullptr) return RBS_ERR_CUDA;
-  const size_t smem = static_cast<size_t>(NW) * B * 256;
-  auto kern = block_stats_warp_kernel<B, NW>;
+  const size_t smem = static_cast<size_t>(NW) * NS * B * 256;
+  auto kern = block_stats_warp_kernel<B, NW, NS>;
   RBS_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   const long long n_tiles = static_cast<long long>(x.L) * x.Hkv * x.M;
   long long want = (n_tiles + NW - 1) / NW;
@@ -151,6 +162,10 @@ extern "C" rbs_status rbs_block_stats(const rbs_shape* shape, rbs_tensor K, rbs_
   const long long n_tiles = static_cast<long long>(x.L) * x.Hkv * x.M;
   if (n_tiles > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (x.B == 256) return launch_stats_warp<256, 3>(K, x, stats, s);
-  return x.B == 128 ? launch_stats_warp<128, 7>(K, x, stats, s) : launch_stats_warp<64, 14>(K, x, stats, s);
+  // Shared memory holds 7 tiles of 32 KB (3 of 64 KB): seven warps with one slot each for B = 128 (three warps with
+  // two slots each were measured compute-bound, 46 us against 32 us per 128K layer), seven warps with two 16 KB
+  // slots each for B = 64 (28.7 us against 31.1 us with fourteen single-slot warps).
+  if (x.B == 256) return launch_stats_warp<256, 3, 1>(K, x, stats, s);
+  if (x.B == 128) return launch_stats_warp<128, 7, 1>(K, x, stats, s);
+  return launch_stats_warp<64, 7, 2>(K, x, stats, s);
 }
