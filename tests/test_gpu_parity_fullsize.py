@@ -86,3 +86,50 @@ def test_fullsize_attention_rows(full):
     err = np.abs(np.concatenate(got) - np.concatenate(want))
     assert err.max() <= 2e-2 and err.mean() <= 2e-3, (err.max(), err.mean())
     assert np.allclose(np.concatenate(got_l), np.concatenate(want_l), atol=2e-3, rtol=1e-4)
+
+
+def test_maximum_block_count():
+    """The largest block count the library accepts (M = 8192; here 512K tokens at block 64, one head): statistics of
+    the whole sequence, complete mask rows of sampled query blocks and their attention rows against the oracle; one
+    block more is refused before anything is launched."""
+    from paper_2609_20971_b200.binding import RbsError
+    from paper_2609_20971_b200.synth import SynthConfig
+    cfg = SynthConfig("max_blocks", N=8192 * 64, Hq=1, Hkv=1, B=64, sigma=0.5, seed=88)
+    M, B = cfg.M, cfg.B
+    assert M == 8192
+    Q, K, V = make_inputs(cfg)
+    dev = torch.device("cuda:0")
+    Qg, Kg, Vg = Q.to(dev), K.to(dev), V.to(dev)
+    stats = rbs_block_stats(Kg, B)
+    mask, dens, mb, mr = rbs_select(Qg, stats, B, cfg.alpha_base, cfg.alpha_rescue, cfg.n_sink, cfg.n_local,
+                                    cfg.n_recent, debug=True)
+    O = rbs_sparse_prefill(Qg, Kg, Vg, mask, B)
+    torch.cuda.synchronize()
+    assert rbs_device_status() == 0
+    K64 = to_f64(K[0, :, 0])
+    c, r = orc.block_stats(K64, B)
+    beta, lo, hi = orc.rescue_coefficient(r)
+    assert np.allclose(stats.centroid[0, 0].cpu().numpy(), c, rtol=2e-5, atol=2e-6)
+    assert np.allclose(stats.radius[0, 0].cpu().numpy(), r, rtol=2e-5)
+    assert np.allclose(stats.beta[0, 0].cpu().numpy(), beta, atol=2e-4)
+    rows = [0, 63, 4097, M - 2, M - 1]
+    Q64, V64 = to_f64(Q[0, :, 0]), to_f64(V[0, :, 0])
+    sel = orc.select_head(Q64, c, r, beta, B, cfg.alpha_base, cfg.alpha_rescue, cfg.n_sink, cfg.n_local, cfg.n_recent,
+                          rows=rows)
+    for i in rows:
+        near = (sel.margin_base[i] <= 1e-3) | (sel.margin_rescue[i] <= 1e-3)
+        got = _row_bits(mask, 0, 0, i, M)
+        assert not ((got != sel.final[i]) & ~near).any()
+        assert not got[i + 1:].any()
+    for i in (63, 4097, M - 2):      # M - 1 is the dense (recent) row: 8192 blocks, left to the smaller cases
+        bits = _row_bits(mask, 0, 0, i, M)
+        o, _ = orc.masked_attention_block(Q64, K64, V64, bits, i, B)
+        err = np.abs(O[0, i * B:(i + 1) * B, 0].float().cpu().numpy() - o)
+        assert err.max() <= 2e-2 and err.mean() <= 2e-3
+    words = mask.cpu().numpy().view(np.uint32)
+    pop = int(np.unpackbits(words.view(np.uint8)).sum())
+    assert abs(float(dens[0, 0]) - pop / (M * (M + 1) / 2)) <= 1e-7
+    # one block more than the maximum
+    one_more = torch.empty(1, (M + 1) * B, 1, 128, dtype=torch.bfloat16, device=dev)
+    with pytest.raises(RbsError, match="UNSUPPORTED"):
+        rbs_block_stats(one_more, B)
