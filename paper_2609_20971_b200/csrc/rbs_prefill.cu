@@ -16,6 +16,7 @@ struct PrefillParams {
   int M, W, L, Hq, G, N;
   int R;   // 128-row tiles per block (tensor-core path): block / 128
   int q0, Mq, Nq;   // this call's queries: first query block (global index), number of blocks, number of tokens
+  int band_rows;    // 128-row query tiles per band of the tile order (tensor-core path)
   float scale_log2;
 };
 
@@ -246,8 +247,9 @@ prefill_mma_kernel(const PrefillParams p) {
 constexpr int kPfThreads = 256;
 constexpr float kRescaleSlack = 8.0f;
 // Of every (kPolyEvery + 1) groups of four logits, one pair is exponentiated by polynomial (0: every group
-// = 50 % of the exps, 1: 25 %, 3: 12.5 %).
-constexpr int kPolyEvery = 1;
+// = 50 % of the exps, 1: 25 %, 3: 12.5 %, 16: none).  Measured on the 128K workload at 8 % density, median of
+// eight launches: 25 % 10.16 ms, 12.5 % 10.02 ms, none 10.06 ms.
+constexpr int kPolyEvery = 3;
 
 __global__ void __launch_bounds__(kPfThreads, 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -265,15 +267,22 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   __shared__ uint32_t s_tmem;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  // Tile order: one (batch, KV head) at a time, inside it longest rows first, the G query heads of the group
+  // Tile order: the query tiles are cut into bands of band_rows consecutive tiles, the last (longest) band first;
+  // inside a band one (batch, KV head) at a time, inside it longest rows first, the G query heads of the group
   // together.  All tiles in flight then read the K/V of one KV head (64 MiB at 128K tokens), which stays in L2;
   // with all KV heads interleaved the K/V tiles of a 128K layer (256 MiB) were re-read from DRAM many times.
+  // The bands keep the very long rows (the dense rows of the last query blocks) of every KV head near the start
+  // of the launch: with one band, the last KV head's dense rows started after three quarters of the launch and
+  // ran on alone after everything else had finished.
   const int R = p.R;
-  const int per_kv = p.Mq * R * p.G;
-  const int kvid = static_cast<int>(blockIdx.x / per_kv), rem = static_cast<int>(blockIdx.x % per_kv);
   const int Hkv = p.Hq / p.G;
+  const int per_band_kv = p.band_rows * p.G;
+  const int per_band = p.L * Hkv * per_band_kv;
+  const int band = static_cast<int>(blockIdx.x / per_band), rem_band = static_cast<int>(blockIdx.x % per_band);
+  const int kvid = rem_band / per_band_kv, rem = rem_band % per_band_kv;
   const int l = kvid / Hkv, hk = kvid % Hkv;
-  const int Tl = p.Mq * R - 1 - rem / p.G;  // 128-row query tile inside this call's chunk
+  const int Tl = p.Mq * R - 1 - (band * p.band_rows + rem / p.G);  // 128-row query tile inside this call's chunk
+  if (Tl < 0) return;                       // padding of the last band
   const int T = p.q0 * R + Tl;              // its position in the sequence (in 128-token units)
   const int i = T / R;                      // its query block
   const int h = hk * p.G + rem % p.G;
@@ -505,9 +514,17 @@ static rbs_status launch_prefill_tc(const PrefillParams& p, const rbs_tensor& Q,
   if (status == nullptr) return RBS_ERR_CUDA;
   const size_t smem = 3 * 2 * 128 * 128;
   RBS_CUDA_OK(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
-  const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.Mq * p.R;
+  PrefillParams pp = p;
+  const int n_rows = p.Mq * p.R;
+  // up to four bands of at least 64 query tiles (512 CTAs per band and KV head at G = 8: enough to fill the GPU
+  // from one KV head).  Measured at 128K, 32 q / 4 kv heads: 1 / 4 / 8 / 16 bands give 5.52 / 4.86 / 4.97 / 4.90 ms
+  // at 3 % density and 17.5 / 16.7 / 17.2 / 17.2 ms at 12 %.
+  int n_bands = n_rows / 64;
+  n_bands = n_bands < 1 ? 1 : (n_bands > 4 ? 4 : n_bands);
+  pp.band_rows = (n_rows + n_bands - 1) / n_bands;
+  const long long n_cta = static_cast<long long>(p.L) * p.Hq * pp.band_rows * n_bands;
   if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
-  prefill_tc_kernel<<<static_cast<unsigned>(n_cta), kPfThreads, smem, s>>>(tmQ, tmK, tmV, p, status);
+  prefill_tc_kernel<<<static_cast<unsigned>(n_cta), kPfThreads, smem, s>>>(tmQ, tmK, tmV, pp, status);
   RBS_CUDA_OK(cudaGetLastError());
   return RBS_OK;
 }
