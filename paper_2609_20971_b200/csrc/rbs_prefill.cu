@@ -241,11 +241,12 @@ prefill_mma_kernel(const PrefillParams p) {
 // thread has read its S row; [128,256) O.
 // Warps 0-3: softmax, one query row per thread (TMEM lane = row).  Warp 4: TMA producer.  Warp 5: MMA issuer.
 // Warps 6-7 only exist so that warps 4-7 form a whole warpgroup that can hand its registers to the softmax warps.
-// The running row maximum is only raised when a block exceeds it by more than kRescaleSlack (log2 units);
-// P then stays below 2^kRescaleSlack and O is rescaled rarely.
+// The running row maximum is lazy: exponentials are taken against the maximum in use and a half-row is redone
+// against its exact maximum only when its sum reaches kSumLimit, so P stays below kSumLimit and O is rescaled rarely.
 // ---------------------------------------------------------------------------------------------
 constexpr int kPfThreads = 256;
-constexpr float kRescaleSlack = 8.0f;
+// A half-row of P whose sum reaches this value makes the row adopt the half's exact maximum.
+constexpr float kSumLimit = 16384.0f;
 // Of every (kPolyEvery + 1) groups of four logits, one pair is exponentiated by polynomial (0: every group
 // = 50 % of the exps, 1: 25 %, 3: 12.5 %, 16: none).  Measured on the 128K workload at 8 % density, median of
 // eight launches: 25 % 10.16 ms, 12.5 % 10.02 ms, none 10.06 ms.
@@ -263,8 +264,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   unsigned char* sQ = smem;
   unsigned char* sK = smem + kTile;
   unsigned char* sV = smem + 2 * kTile;
-  __shared__ __align__(8) uint64_t bar_q, bar_kfull, bar_vfull, bar_s, bar_p, bar_p1, bar_pv;
+  __shared__ __align__(8) uint64_t bar_q, bar_kfull, bar_vfull, bar_s, bar_p, bar_p1, bar_pv0, bar_pv;
   __shared__ uint32_t s_tmem;
+  // Per key sub-block, written by the MMA warp before it issues S = Q K^T of that block (two entries used in turn):
+  // bit 0: the block is the diagonal one; bit 1: it is the tile's last block.  The softmax warps read it instead of
+  // walking the mask themselves.
+  __shared__ uint32_t s_blk[2];
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   // Tile order: the query tiles are cut into bands of band_rows consecutive tiles, the last (longest) band first;
@@ -296,6 +301,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     mbar_init(smem_u32(&bar_s), 1);
     mbar_init(smem_u32(&bar_p), 128);
     mbar_init(smem_u32(&bar_p1), 128);
+    mbar_init(smem_u32(&bar_pv0), 1);
     mbar_init(smem_u32(&bar_pv), 1);
     mbar_fence_init();
   }
@@ -341,23 +347,31 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       const uint64_t dq = smem_desc_sw128(smem_u32(sQ), 16, 1024);
       const uint64_t dk = smem_desc_sw128(smem_u32(sK), 16, 1024);
       const uint64_t dv = smem_desc_sw128(smem_u32(sV), kPanel, 1024);
-      auto issue_qk = [&]() { mma_ss_k128_commit_elect(tmem_s, dq, dk, kIdescQK, kPanel, kPanel, smem_u32(&bar_s)); };
+      auto issue_qk = [&](int j, int blk, int blk_next) {
+        if (lane == 0) {
+          s_blk[j & 1] = (blk == T ? 1u : 0u) | (blk_next < 0 ? 2u : 0u);
+          __threadfence_block();
+        }
+        __syncwarp();
+        mma_ss_k128_commit_elect(tmem_s, dq, dk, kIdescQK, kPanel, kPanel, smem_u32(&bar_s));
+      };
+      int b_next = b >= 0 ? next_kb(mrow, b, i, R, T) : -1;
       ok = __all_sync(0xffffffffu, ok);
       if (ok && b >= 0) {
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull), 0, status, kWaitTmaFull));
         if (ok) {
           tc_fence_after_sync();
-          issue_qk();
+          issue_qk(0, b, b_next);
         }
       }
       for (int j = 0; ok && b >= 0; ++j) {
         const uint32_t ph = j & 1;
-        const int b_next = next_kb(mrow, b, i, R, T);     // global-memory latency hidden behind the softmax
+        const int b_next2 = b_next >= 0 ? next_kb(mrow, b_next, i, R, T) : -1;   // global-memory latency hidden behind the softmax
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_vfull), ph, status, kWaitTmaFull) &&
                                          mbar_wait(smem_u32(&bar_p), ph, status, kWaitPReady));   // P of keys 0..63
         if (!ok) break;
         tc_fence_after_sync();
-        mma_ts_k64_elect(tmem_o, tmem_s, dv, kIdescPV, 2048 >> 4, j != 0, 0);
+        mma_ts_k64_elect(tmem_o, tmem_s, dv, kIdescPV, 2048 >> 4, j != 0, smem_u32(&bar_pv0));
         // K of the next block arrived while the softmax ran; checking it here, before the wait for the second half
         // of P, keeps that check (about 200 cycles of wait, vote and fence) off the tile's critical path
         if (b_next >= 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull), ph ^ 1, status, kWaitTmaFull));
@@ -365,8 +379,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         if (!ok) break;
         tc_fence_after_sync();
         mma_ts_k64_elect(tmem_o, tmem_s + 32, dv + static_cast<uint64_t>((4 * 2048) >> 4), kIdescPV, 2048 >> 4, 1, smem_u32(&bar_pv));
-        if (b_next >= 0) issue_qk();
+        if (b_next >= 0) issue_qk(j + 1, b_next, b_next2);
         b = b_next;
+        b_next = b_next2;
       }
     }
     __syncwarp();
@@ -381,8 +396,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     bool ok = true;
     int j = 0;
     const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
-    for (; b >= 0; ++j, b = next_kb(mrow, b, i, R, T)) {
+    for (bool more = any_block; more; ++j) {
       if (!(ok = mbar_wait(smem_u32(&bar_s), j & 1, status, kWaitMmaDone))) break;
+      const uint32_t blk = *reinterpret_cast<volatile uint32_t*>(&s_blk[j & 1]);
+      more = (blk & 2u) == 0u;
       tc_fence_after_sync();
       uint32_t s[128];   // the whole S row of this thread
       {
@@ -396,75 +413,87 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         tmem_ld32(tmem_s + lane_off + 96, s3);
         tmem_wait_ld();
       }
-      if (b == T) {   // diagonal sub-block: keys after the query are hidden
+      if (blk & 1u) {   // diagonal sub-block: keys after the query are hidden
 #pragma unroll
         for (int c = 0; c < 128; ++c)
           if (c > row) s[c] = 0xff800000u;   // -inf
       }
-      float mxa[8];
-#pragma unroll
-      for (int u = 0; u < 8; ++u) mxa[u] = -INFINITY;
-#pragma unroll
-      for (int c = 0; c < 128; c += 16) {
-#pragma unroll
-        for (int u = 0; u < 8; ++u) mxa[u] = max3(mxa[u], __uint_as_float(s[c + 2 * u]), __uint_as_float(s[c + 2 * u + 1]));
-      }
-      const float mx = fmaxf(max3(mxa[0], mxa[1], mxa[2]), max3(max3(mxa[3], mxa[4], mxa[5]), mxa[6], mxa[7])) * p.scale_log2;
-      const bool raise = mx > m_used + kRescaleSlack;     // always true for the first block (m_used = -inf)
-      if (__any_sync(0xffffffffu, raise)) {
-        const float m_new = raise ? mx : m_used;
-        const float corr = fast_exp2(m_used - m_new);     // 0 for the first block
-        l_sum *= corr;
-        m_used = m_new;
-        if (j > 0) {
-          if (!(ok = mbar_wait(smem_u32(&bar_pv), (j - 1) & 1, status, kWaitOReady))) break;
-          tc_fence_after_sync();
-#pragma unroll
-          for (int c0 = 0; c0 < 128; c0 += 32) {
-            uint32_t r[32];
-            tmem_ld32(tmem_o + lane_off + c0, r);
-            tmem_wait_ld();
-#pragma unroll
-            for (int q = 0; q < 32; ++q) r[q] = __float_as_uint(__uint_as_float(r[q]) * corr);
-            tmem_st32(tmem_o + lane_off + c0, r);
-          }
-        }
-      }
-      const uint64_t negm2 = f2_pack(-m_used, -m_used);
-      uint64_t sum_a = 0ull, sum_b = 0ull;   // (0.f, 0.f)
+      // Lazy running maximum: the exponentials of a half are first taken against the maximum in use.  Only when a
+      // half's sum shows that this has gone stale (sum >= kSumLimit, or not finite; always so for the very first
+      // half, where the maximum is still -inf) is the exact maximum of the half computed, O and l rescaled and
+      // the half redone.  The maximum is a shift that cancels in O / l, so any value that keeps P finite is right.
 #pragma unroll
       for (int half = 0; half < 2; ++half) {
         uint32_t pk[32];
+        auto exps = [&]() -> float {
+          const uint64_t negm2 = f2_pack(-m_used, -m_used);
+          uint64_t sum_a = 0ull, sum_b = 0ull;   // (0.f, 0.f)
 #pragma unroll
-        for (int q = 0; q < 64; q += 4) {
-          const int c = half * 64 + q;
-          const uint64_t x01 = f2_fma(f2_pack(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), scale2, negm2);
-          const uint64_t x23 = f2_fma(f2_pack(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), scale2, negm2);
-          float x0, x1, x2, x3;
-          f2_unpack(x01, x0, x1);
-          f2_unpack(x23, x2, x3);
-          const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
-          float p2, p3;
-          if (((q >> 2) & kPolyEvery) == kPolyEvery) {   // a share of the exps goes to the FMA pipe
-            exp2_poly_x2(x23, p2, p3);
-          } else {
-            p2 = fast_exp2(x2);
-            p3 = fast_exp2(x3);
+          for (int q = 0; q < 64; q += 4) {
+            const int c = half * 64 + q;
+            const uint64_t x01 = f2_fma(f2_pack(__uint_as_float(s[c]), __uint_as_float(s[c + 1])), scale2, negm2);
+            const uint64_t x23 = f2_fma(f2_pack(__uint_as_float(s[c + 2]), __uint_as_float(s[c + 3])), scale2, negm2);
+            float x0, x1, x2, x3;
+            f2_unpack(x01, x0, x1);
+            f2_unpack(x23, x2, x3);
+            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1);
+            float p2, p3;
+            if (((q >> 2) & kPolyEvery) == kPolyEvery) {   // a share of the exps goes to the FMA pipe
+              exp2_poly_x2(x23, p2, p3);
+            } else {
+              p2 = fast_exp2(x2);
+              p3 = fast_exp2(x3);
+            }
+            sum_a = f2_add(sum_a, f2_pack(p0, p1));
+            sum_b = f2_add(sum_b, f2_pack(p2, p3));
+            pk[q >> 1] = pack_bf16(p0, p1);
+            pk[(q >> 1) + 1] = pack_bf16(p2, p3);
           }
-          sum_a = f2_add(sum_a, f2_pack(p0, p1));
-          sum_b = f2_add(sum_b, f2_pack(p2, p3));
-          pk[q >> 1] = pack_bf16(p0, p1);
-          pk[(q >> 1) + 1] = pack_bf16(p2, p3);
+          float a0, a1, a2, a3;
+          f2_unpack(sum_a, a0, a1);
+          f2_unpack(sum_b, a2, a3);
+          return (a0 + a1) + (a2 + a3);
+        };
+        float hs = exps();
+        if (__any_sync(0xffffffffu, !(hs < kSumLimit))) {
+          float mxa[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) mxa[u] = -INFINITY;
+#pragma unroll
+          for (int c = half * 64; c < half * 64 + 64; c += 8) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) mxa[u] = max3(mxa[u], __uint_as_float(s[c + 2 * u]), __uint_as_float(s[c + 2 * u + 1]));
+          }
+          const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])) * p.scale_log2;
+          const float m_new = fmaxf(m_used, mx);
+          const float corr = fast_exp2(m_used - m_new);     // 0 while m_used = -inf
+          l_sum *= corr;
+          m_used = m_new;
+          if (j > 0 || half > 0) {   // O holds the P V of everything issued so far: wait for it, then rescale
+            if (ok) ok = half == 0 ? mbar_wait(smem_u32(&bar_pv), (j - 1) & 1, status, kWaitOReady)
+                                   : mbar_wait(smem_u32(&bar_pv0), j & 1, status, kWaitOReady);
+            if (ok) {
+              tc_fence_after_sync();
+#pragma unroll
+              for (int c0 = 0; c0 < 128; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(tmem_o + lane_off + c0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int q = 0; q < 32; ++q) r[q] = __float_as_uint(__uint_as_float(r[q]) * corr);
+                tmem_st32(tmem_o + lane_off + c0, r);
+              }
+            }
+          }
+          hs = exps();
         }
+        l_sum += hs;
         tmem_st32(tmem_s + lane_off + half * 32, pk);
         tmem_wait_st();
         tc_fence_before_sync();
         mbar_arrive(smem_u32(half == 0 ? &bar_p : &bar_p1));
       }
-      float a0, a1, a2, a3;
-      f2_unpack(sum_a, a0, a1);
-      f2_unpack(sum_b, a2, a3);
-      l_sum += (a0 + a1) + (a2 + a3);
+      if (!ok) break;
     }
     // epilogue: O / l -> bf16 -> global
     __nv_bfloat16* orow = p.O + l * p.osb + (static_cast<int64_t>(Tl) * B + row) * p.ost + h * p.osh;

@@ -415,3 +415,28 @@ def test_varlen_batch_equals_one_call_per_prompt():
     ref, _ = orc.dense_causal_attention(Q64[0, :, 0], K64[0, :, 0], V64[0, :, 0])
     got = O[cu[k]:cu[k + 1], 0].float().cpu().numpy()
     assert np.abs(got - ref).max() <= OUT_MAX_ABS
+
+
+@pytest.mark.parametrize("pos", [10, 100])
+def test_logit_jump_inside_a_block(pos):
+    """One key far out of scale (its logit exceeds everything before it by about 115 in log2 units) in the first or
+    the second half of a late key block: the running maximum has to be replaced in the middle of the block and O
+    rescaled, for the rows that see the key and only for them."""
+    dev = torch.device("cuda:0")
+    B, N, d = 128, 128 * 6, 128
+    g = torch.Generator().manual_seed(91 + pos)
+    u = torch.ones(d) / math.sqrt(d)
+    Q = (3.0 * u + 0.5 * torch.randn(N, d, generator=g)).to(torch.bfloat16).view(1, N, 1, d)
+    K = (0.1 * torch.randn(N, d, generator=g))
+    t_big = 3 * B + pos
+    K[t_big] = 300.0 * u
+    K = K.to(torch.bfloat16).view(1, N, 1, d)
+    V = torch.randn(N, d, generator=g).to(torch.bfloat16).view(1, N, 1, d)
+    O, lse = rbs_sparse_prefill(Q.to(dev), K.to(dev), V.to(dev), None, B, return_lse=True)
+    torch.cuda.synchronize()
+    ref, ref_lse = orc.dense_causal_attention(to_f64(Q[0, :, 0]), to_f64(K[0, :, 0]), to_f64(V[0, :, 0]))
+    err = np.abs(O[0, :, 0].float().cpu().numpy() - ref)
+    assert err.max() <= OUT_MAX_ABS and err.mean() <= OUT_MEAN_ABS, (err.max(), err.mean())
+    assert np.allclose(lse[0, 0].cpu().numpy(), ref_lse, atol=2e-3, rtol=1e-4)
+    # rows from the big key on are its value row (to bf16 rounding); earlier rows are not
+    assert np.abs(O[0, t_big + 5, 0].float().cpu().numpy() - V[0, t_big, 0].float().numpy()).max() <= 2e-2
