@@ -440,3 +440,23 @@ def test_logit_jump_inside_a_block(pos):
     assert np.allclose(lse[0, 0].cpu().numpy(), ref_lse, atol=2e-3, rtol=1e-4)
     # rows from the big key on are its value row (to bf16 rounding); earlier rows are not
     assert np.abs(O[0, t_big + 5, 0].float().cpu().numpy() - V[0, t_big, 0].float().numpy()).max() <= 2e-2
+
+
+def test_whole_path_is_bitwise_repeatable():
+    """Statistics, selection and attention (sparse and dense) give bit-identical results launch after launch:
+    nothing in the path depends on the order in which CTAs happen to run."""
+    dev = torch.device("cuda:0")
+    cfg = SynthConfig("repeat", N=128 * 37 + 55, Hq=8, Hkv=2, B=128, sigma=(0.1, 1.0), seed=5)
+    Q, K, V = (t.to(dev) for t in make_inputs(cfg))
+    ref = None
+    for _ in range(25):
+        st = rbs_block_stats(K, cfg.B)
+        mask, dens = rbs_select(Q, st, cfg.B, cfg.alpha_base, cfg.alpha_rescue, cfg.n_sink, cfg.n_local, cfg.n_recent)
+        O = rbs_sparse_prefill(Q, K, V, mask, cfg.B)
+        Od = rbs_sparse_prefill(Q, K, V, None, cfg.B)
+        torch.cuda.synchronize()
+        cur = (st.centroid, st.radius, st.beta, mask, dens, O, Od)
+        if ref is None:
+            ref = cur
+        else:
+            assert all(torch.equal(a, b) for a, b in zip(ref, cur))
