@@ -388,7 +388,9 @@ def run_ours(args):
         "roofline": {"bound": "tensor", "kernel": "rbs_sparse_prefill", "achieved": tflops_sparse,
                      "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": tflops_sparse / peaks["tflops"],
                      "traffic": NCU_TRAFFIC_BYTES.get(cfg.name), "algorithmic_bytes": int(2 * Qg.numel() * 2 + 2 * Kg.numel() * 2 + mask.numel() * 4),
-                     "peak_source": peaks["source"],
+                     "peak_source": peaks["source"], "peak_kind": "burst (the timed region is ten short steps)",
+                     "peak_sustained": peaks.get("tflops_sustained"),
+                     "frac_of_sustained": (tflops_sparse / peaks["tflops_sustained"]) if peaks.get("tflops_sustained") else None,
                      "flops_per_launch_useful": useful, "flops_per_launch_executed": executed},
         "cpu_baseline": ({"value": cpu_ms, "unit": UNIT, "cores": torch.get_num_threads(), "kind": "oracle",
                           "sample": cpu_sample, "parts": cpu_parts} if cpu_ms is not None else None),
