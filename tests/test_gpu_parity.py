@@ -460,3 +460,32 @@ def test_whole_path_is_bitwise_repeatable():
             ref = cur
         else:
             assert all(torch.equal(a, b) for a, b in zip(ref, cur))
+
+
+def test_batch_stride_beyond_32_bits():
+    """Two layers whose data sit more than 2^31 elements apart inside one buffer (strided views, nothing copied):
+    every kernel must carry the batch offset in 64 bits.  Checked bit for bit against the same data held contiguously."""
+    dev = torch.device("cuda:0")
+    B, N, Hq, Hkv, d = 128, 128 * 9 + 40, 4, 2, 128
+    SB = (1 << 31) + (1 << 20)                       # batch stride in elements
+    nq, nk = N * Hq * d, N * Hkv * d
+    big = torch.empty(SB + 2 * nq + 2 * nk, dtype=torch.bfloat16, device=dev)
+
+    def view(off, H):
+        return torch.as_strided(big, (2, N, H, d), (SB, H * d, d, 1), off)
+    Qv, Ov = view(0, Hq), view(nq, Hq)
+    Kv, Vv = view(2 * nq, Hkv), view(2 * nq + nk, Hkv)
+    cfg = SynthConfig("stride", L=2, N=N, Hq=Hq, Hkv=Hkv, B=B, sigma=(0.1, 1.0), seed=77)
+    Q, K, V = (t.to(dev) for t in make_inputs(cfg))
+    Qv.copy_(Q); Kv.copy_(K); Vv.copy_(V)
+    st_v = rbs_block_stats(Kv, B)
+    mask_v, dens_v = rbs_select(Qv, st_v, B)
+    rbs_sparse_prefill(Qv, Kv, Vv, mask_v, B, out=Ov)
+    st = rbs_block_stats(K, B)
+    mask, dens = rbs_select(Q, st, B)
+    O = rbs_sparse_prefill(Q, K, V, mask, B)
+    torch.cuda.synchronize()
+    assert torch.equal(st_v.centroid, st.centroid) and torch.equal(st_v.radius, st.radius)
+    assert torch.equal(mask_v, mask) and torch.equal(dens_v, dens)
+    assert torch.equal(Ov, O)
+    assert not torch.equal(O[0], O[1])               # the two layers really differ
