@@ -13,30 +13,41 @@ namespace rbs {
 // Pass 2: lanes own rows and walk the columns (row distances, no cross-lane traffic); the swizzle
 // keeps both access patterns free of bank conflicts.
 // ---------------------------------------------------------------------------------------------
-template <int B, int NW, int NS>
+// With WPB = 2 (blocks of 256) two neighbouring warps share a block, 128 rows each: they exchange their column
+// sums and their row maxima through shared memory (two bounded mbarrier rendezvous per block), so a block of 256
+// streams like two blocks of 128 instead of needing a 64 KB slot per warp.
+template <int B, int NW, int NS, int WPB>
 __global__ void __launch_bounds__(NW * 32, 1)
 block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, int M, int Hkv, int N,
                         float* __restrict__ centroid, float* __restrict__ radius, unsigned int* status) {
-  constexpr uint32_t kPanel = B * 128;       // bytes of one 64-column panel
+  constexpr int RW = B / WPB;                 // rows of a block held by one warp
+  constexpr uint32_t kPanel = RW * 128;      // bytes of one 64-column panel
   constexpr uint32_t kSlot = 2 * kPanel;
-  constexpr int RJ = B / 32;                  // rows per lane in pass 2
+  constexpr int RJ = RW / 32;                 // rows per lane in pass 2
+  constexpr int NG = NW / WPB;                // blocks in flight per CTA
+  static_assert(NW % WPB == 0 && (WPB == 1 || WPB == 2), "warps per block");
   extern __shared__ __align__(1024) unsigned char smem[];
   __shared__ __align__(8) uint64_t full_bar[NW * NS];
   // half of the warp's centroid (64 columns) at a time, re-read by every lane in pass 2; the whole of it would not
   // fit beside the tile slots
   __shared__ __align__(16) float s_cen[NW][kHeadDim / 2];
+  __shared__ __align__(16) float s_sum[WPB == 2 ? NW : 1][kHeadDim];   // a warp's column sums, for its partner
+  __shared__ float s_max[WPB == 2 ? NW : 1];
+  __shared__ __align__(8) uint64_t pair_bar[NG];
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const uint32_t bar0 = smem_u32(&full_bar[warp * NS]);
   const uint32_t slot0 = smem_u32(smem) + warp * NS * kSlot;
+  const int group = warp / WPB, part = warp % WPB;
   if (lane == 0) {
     for (int k = 0; k < NS; ++k) mbar_init(bar0 + 8 * k, 1);
+    if (WPB == 2 && part == 0) mbar_init(smem_u32(&pair_bar[group]), 64);
     mbar_fence_init();
   }
-  __syncwarp();
+  if (WPB == 2) __syncthreads(); else __syncwarp();
 
-  const int stride = gridDim.x * NW;
-  int t = warp * gridDim.x + blockIdx.x;
+  const int stride = gridDim.x * NG;
+  int t = group * gridDim.x + blockIdx.x;
   auto issue = [&](int tile, int buf) {
     const uint32_t bar = bar0 + 8 * buf, slot = slot0 + buf * kSlot;
     int idx = tile;
@@ -44,8 +55,8 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
     const int b = idx % M;
     const int l = idx / M;
     mbar_arrive_expect_tx(bar, kSlot);
-    tma_load_4d(slot, &tmK, bar, 0, hk, b * B, l);
-    tma_load_4d(slot + kPanel, &tmK, bar, 64, hk, b * B, l);
+    tma_load_4d(slot, &tmK, bar, 0, hk, b * B + part * RW, l);
+    tma_load_4d(slot + kPanel, &tmK, bar, 64, hk, b * B + part * RW, l);
   };
   if (lane == 0) {
     for (int k = 0; k < NS; ++k)
@@ -62,7 +73,7 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
     if (!mbar_wait(bar0 + 8 * buf, phase, status, kWaitTmaFull)) break;
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll 4
-    for (int r8 = 0; r8 < B; r8 += 8) {
+    for (int r8 = 0; r8 < RW; r8 += 8) {
 #pragma unroll
       for (int rr = 0; rr < 8; ++rr) {
         uint32_t lo, hi;
@@ -76,11 +87,20 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
     const int b = idx % M;
     const int l = idx / M;
     // a short last block: TMA filled the rows past the sequence end with zeros; divide by its own size |K_b|
-    const int rows_valid = min(B, N - b * B);
-    const float inv_rows = 1.0f / static_cast<float>(rows_valid);
+    const int rows_block = min(B, N - b * B);
+    const int rows_valid = max(0, min(RW, rows_block - part * RW));   // of this warp's rows
+    const float inv_rows = 1.0f / static_cast<float>(rows_block);
+    bool pair_ok = true;
+    if (WPB == 2) {   // add the partner's column sums (rows past the sequence end arrived as zeros)
+      reinterpret_cast<float4*>(s_sum[warp])[lane] = make_float4(a0, a1, a2, a3);
+      mbar_arrive(smem_u32(&pair_bar[group]));
+      pair_ok = mbar_wait(smem_u32(&pair_bar[group]), 0, status, kWaitStageFree);
+      const float4 o = reinterpret_cast<const float4*>(s_sum[warp ^ 1])[lane];
+      a0 += o.x; a1 += o.y; a2 += o.z; a3 += o.w;
+    }
     const float4 cen = make_float4(a0 * inv_rows, a1 * inv_rows, a2 * inv_rows, a3 * inv_rows);
     const int64_t blk = (static_cast<int64_t>(l) * Hkv + hk) * M + b;
-    reinterpret_cast<float4*>(centroid + blk * kHeadDim)[lane] = cen;
+    if (part == 0) reinterpret_cast<float4*>(centroid + blk * kHeadDim)[lane] = cen;
 
     float q[RJ];
 #pragma unroll
@@ -125,23 +145,31 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) rmax = fmaxf(rmax, __shfl_xor_sync(0xffffffffu, rmax, o));
-    if (lane == 0) radius[blk] = sqrtf(rmax);
+    if (WPB == 2) {
+      if (lane == 0) s_max[warp] = rmax;
+      mbar_arrive(smem_u32(&pair_bar[group]));
+      pair_ok = mbar_wait(smem_u32(&pair_bar[group]), 1, status, kWaitStageFree) && pair_ok;
+      if (part == 0 && lane == 0) radius[blk] = sqrtf(fmaxf(rmax, s_max[warp ^ 1]));
+      if (!__all_sync(0xffffffffu, pair_ok)) break;
+    } else {
+      if (lane == 0) radius[blk] = sqrtf(rmax);
+    }
   }
 }
 
-template <int B, int NW, int NS>
+template <int B, int NW, int NS, int WPB>
 static rbs_status launch_stats_warp(const rbs_tensor& K, const Dims& x, const rbs_stats& stats, cudaStream_t s) {
   CUtensorMap tm;
   rbs_status st = make_tmap_lthd(&tm, K.ptr, x.L, x.N, x.Hkv, x.d, K.stride_batch, K.stride_token, K.stride_head,
-                                 64, B, true);
+                                 64, B / WPB, true);
   if (st != RBS_OK) return st;
   unsigned int* status = device_status_ptr();
   if (status == nullptr) return RBS_ERR_CUDA;
-  const size_t smem = static_cast<size_t>(NW) * NS * B * 256;
-  auto kern = block_stats_warp_kernel<B, NW, NS>;
+  const size_t smem = static_cast<size_t>(NW) * NS * (B / WPB) * 256;
+  auto kern = block_stats_warp_kernel<B, NW, NS, WPB>;
   RBS_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
   const long long n_tiles = static_cast<long long>(x.L) * x.Hkv * x.M;
-  long long want = (n_tiles + NW - 1) / NW;
+  long long want = (n_tiles + NW / WPB - 1) / (NW / WPB);
   const int grid = static_cast<int>(want < sm_count() ? want : sm_count());
   kern<<<grid, NW * 32, smem, s>>>(tm, static_cast<int>(n_tiles), x.M, x.Hkv, x.N, stats.centroid, stats.radius, status);
   RBS_CUDA_OK(cudaGetLastError());
@@ -165,7 +193,7 @@ extern "C" rbs_status rbs_block_stats(const rbs_shape* shape, rbs_tensor K, rbs_
   // Shared memory holds 7 tiles of 32 KB (3 of 64 KB): seven warps with one slot each for B = 128 (three warps with
   // two slots each were measured compute-bound, 46 us against 32 us per 128K layer), seven warps with two 16 KB
   // slots each for B = 64 (28.7 us against 31.1 us with fourteen single-slot warps).
-  if (x.B == 256) return launch_stats_warp<256, 3, 1>(K, x, stats, s);
-  if (x.B == 128) return launch_stats_warp<128, 7, 1>(K, x, stats, s);
-  return launch_stats_warp<64, 7, 2>(K, x, stats, s);
+  if (x.B == 256) return launch_stats_warp<256, 6, 1, 2>(K, x, stats, s);
+  if (x.B == 128) return launch_stats_warp<128, 7, 1, 1>(K, x, stats, s);
+  return launch_stats_warp<64, 7, 2, 1>(K, x, stats, s);
 }
