@@ -190,10 +190,12 @@ extern "C" rbs_status rbs_block_stats(const rbs_shape* shape, rbs_tensor K, rbs_
   const long long n_tiles = static_cast<long long>(x.L) * x.Hkv * x.M;
   if (n_tiles > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  // Shared memory holds 7 tiles of 32 KB (3 of 64 KB): seven warps with one slot each for B = 128 (three warps with
-  // two slots each were measured compute-bound, 46 us against 32 us per 128K layer), seven warps with two 16 KB
-  // slots each for B = 64 (28.7 us against 31.1 us with fourteen single-slot warps).
+  // Shared memory holds 6 or 7 tiles of 32 KB.  Measured per 128K layer of 4 KV heads (128 MiB):
+  //   B = 128: twelve warps in pairs, 64 rows and a 16 KB slot each   31.2 us   (seven warps, one 32 KB slot each:
+  //            32.4 us; three warps with two 32 KB slots each: 46 us, compute-bound)
+  //   B = 64:  seven warps with two 16 KB slots each used in turn      28.7 us   (fourteen single-slot warps: 31.1 us)
+  //   B = 256: six warps in pairs, 128 rows and a 32 KB slot each      35.7 us   (three warps, 64 KB slots: 58 us)
   if (x.B == 256) return launch_stats_warp<256, 6, 1, 2>(K, x, stats, s);
-  if (x.B == 128) return launch_stats_warp<128, 7, 1, 1>(K, x, stats, s);
+  if (x.B == 128) return launch_stats_warp<128, 12, 1, 2>(K, x, stats, s);
   return launch_stats_warp<64, 7, 2, 1>(K, x, stats, s);
 }
