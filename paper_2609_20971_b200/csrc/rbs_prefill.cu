@@ -254,7 +254,8 @@ constexpr int kPolyEvery = 3;
 
 __global__ void __launch_bounds__(kPfThreads, 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
-                  const __grid_constant__ CUtensorMap tmV, const PrefillParams p, unsigned int* status) {
+                  const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                  const PrefillParams p, unsigned int* status) {
   constexpr int B = 128;
   constexpr uint32_t kPanel = B * 128;   // 16 KB: 128 rows x 64 bf16 columns
   constexpr uint32_t kTile = 2 * kPanel;
@@ -505,11 +506,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         for (int c = 0; c < 16; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
         if (lse_dst) *lse_dst = -INFINITY;
       }
-    } else if (ok && mbar_wait(smem_u32(&bar_pv), (j - 1) & 1, status, kWaitOReady)) {
+    } else {
+      // every thread of the four warps reaches the barrier below, also one whose wait has given up
+      const bool o_ready = __all_sync(0xffffffffu, ok && mbar_wait(smem_u32(&bar_pv), (j - 1) & 1, status, kWaitOReady));
+      // O / l -> bf16 -> the Q buffer (free since the tile's last Q K^T), in the swizzled layout of a 128-byte-swizzle
+      // tensor map, then two TMA stores: whole 128-byte lines go out instead of one 16-byte piece per row and
+      // instruction, and rows past the end of the sequence are clipped by the tensor map.
       tc_fence_after_sync();
       const float inv = 1.0f / l_sum;
+      const uint32_t srow = smem_u32(sQ) + row * 128;
 #pragma unroll
-      for (int c0 = 0; c0 < 128; c0 += 32) {
+      for (int c0 = 0; o_ready && c0 < 128; c0 += 32) {
         uint32_t r[32];
         tmem_ld32(tmem_o + lane_off + c0, r);
         tmem_wait_ld();
@@ -520,10 +527,20 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           v.y = pack_bf16(__uint_as_float(r[q + 2]) * inv, __uint_as_float(r[q + 3]) * inv);
           v.z = pack_bf16(__uint_as_float(r[q + 4]) * inv, __uint_as_float(r[q + 5]) * inv);
           v.w = pack_bf16(__uint_as_float(r[q + 6]) * inv, __uint_as_float(r[q + 7]) * inv);
-          if (in_seq) *reinterpret_cast<uint4*>(orow + c0 + q) = v;
+          const int chunk = (c0 + q) >> 3;   // 16-byte piece 0..15 of the row
+          const uint32_t dst = srow + (chunk >> 3) * kPanel + (((chunk & 7) ^ (row & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
         }
       }
-      if (lse_dst && in_seq) *lse_dst = (m_used + fast_log2(l_sum)) * 0.6931471805599453f;
+      fence_proxy_async_smem();
+      asm volatile("bar.sync 1, 128;" ::: "memory");   // the four softmax warps
+      if (tid == 0 && o_ready) {
+        tma_store_4d(&tmO, smem_u32(sQ), 0, h, Tl * B, l);
+        tma_store_4d(&tmO, smem_u32(sQ + kPanel), 64, h, Tl * B, l);
+        tma_store_commit();
+        tma_store_wait_read();
+      }
+      if (lse_dst && in_seq && o_ready) *lse_dst = (m_used + fast_log2(l_sum)) * 0.6931471805599453f;
     }
   }
   tc_fence_before_sync();
@@ -539,6 +556,9 @@ static rbs_status launch_prefill_tc(const PrefillParams& p, const rbs_tensor& Q,
   if ((st = make_tmap_lthd(&tmQ, Q.ptr, p.L, p.Nq, p.Hq, kHeadDim, Q.stride_batch, Q.stride_token, Q.stride_head, 64, 128, true)) != RBS_OK) return st;
   if ((st = make_tmap_lthd(&tmK, K.ptr, p.L, p.N, Hkv, kHeadDim, K.stride_batch, K.stride_token, K.stride_head, 64, 128, true)) != RBS_OK) return st;
   if ((st = make_tmap_lthd(&tmV, V.ptr, p.L, p.N, Hkv, kHeadDim, V.stride_batch, V.stride_token, V.stride_head, 64, 128, true)) != RBS_OK) return st;
+  CUtensorMap tmO;
+  const int64_t osb = p.osb, ost = p.ost, osh = p.osh;
+  if ((st = make_tmap_lthd(&tmO, p.O, p.L, p.Nq, p.Hq, kHeadDim, osb, ost, osh, 64, 128, true)) != RBS_OK) return st;
   unsigned int* status = device_status_ptr();
   if (status == nullptr) return RBS_ERR_CUDA;
   const size_t smem = 3 * 2 * 128 * 128;
@@ -553,7 +573,7 @@ static rbs_status launch_prefill_tc(const PrefillParams& p, const rbs_tensor& Q,
   pp.band_rows = (n_rows + n_bands - 1) / n_bands;
   const long long n_cta = static_cast<long long>(p.L) * p.Hq * pp.band_rows * n_bands;
   if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
-  prefill_tc_kernel<<<static_cast<unsigned>(n_cta), kPfThreads, smem, s>>>(tmQ, tmK, tmV, pp, status);
+  prefill_tc_kernel<<<static_cast<unsigned>(n_cta), kPfThreads, smem, s>>>(tmQ, tmK, tmV, tmO, pp, status);
   RBS_CUDA_OK(cudaGetLastError());
   return RBS_OK;
 }
