@@ -247,10 +247,12 @@ prefill_mma_kernel(const PrefillParams p) {
 constexpr int kPfThreads = 256;
 // A half-row of P whose sum reaches this value makes the row adopt the half's exact maximum.
 constexpr float kSumLimit = 16384.0f;
-// Of every (kPolyEvery + 1) groups of four logits, one pair is exponentiated by polynomial (0: every group
-// = 50 % of the exps, 1: 25 %, 3: 12.5 %, 16: none).  Measured on the 128K workload at 8 % density, median of
-// eight launches: 25 % 10.16 ms, 12.5 % 10.02 ms, none 10.06 ms.
-constexpr int kPolyEvery = 3;
+// Of every (kPolyEvery + 1) groups of four logits, one pair is exponentiated by polynomial on the FMA pipe instead of
+// by ex2 (0: every group = 50 % of the exps, 1: 25 %, 3: 12.5 %, 16: none).  The polynomial relieves the exp unit but
+// costs about six instructions per element, and the launch is bound by power, not by the exp unit: on the 128K
+// workload at 8 % density (median burst / back-to-back ms) 25 %: 10.12 / 11.56, 12.5 %: 10.02 / 11.44, none:
+// 9.89 / 11.32.
+constexpr int kPolyEvery = 16;
 
 __global__ void __launch_bounds__(kPfThreads, 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
