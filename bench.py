@@ -28,7 +28,7 @@ import torch
 
 # DRAM bytes (read + write) of one rbs_sparse_prefill launch from an ncu capture of that workload at the default
 # thresholds (profiles/prefill_tc_kernel_traffic_q30b_128k.md); None where no capture of that workload exists.
-NCU_TRAFFIC_BYTES = {"q30b_128k": 4625449472 + 1049334528}
+NCU_TRAFFIC_BYTES = {"q30b_128k": 4552352512 + 1036708096}
 
 METRIC = "prefill_attention_ms_per_layer_128k"
 UNIT = "ms/layer"
