@@ -254,7 +254,7 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       if (exact_shift) {
       // pass 1: maxima of the raw logits x and of y = x + ||q|| r beta
       float mb0 = -INFINITY, mb1 = -INFINITY, mr0 = -INFINITY, mr1 = -INFINITY;
-#pragma unroll
+#pragma unroll 1
       for (int c0 = 0; c0 < B; c0 += 32) {
         uint32_t r[32];
         tmem_ld32(taddr + c0, r);
@@ -281,7 +281,7 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
       }
       const uint64_t nmb2 = f2_pack(-mb, -mb), nmr2 = f2_pack(-mr, -mr);
       uint64_t sb2 = 0ull, sr2 = 0ull, sb2b = 0ull, sr2b = 0ull;
-#pragma unroll
+#pragma unroll 1
       for (int c0 = 0; c0 < B; c0 += 32) {
         uint32_t r[32];
         tmem_ld32(taddr + c0, r);
