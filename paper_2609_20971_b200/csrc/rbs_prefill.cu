@@ -457,8 +457,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
           f2_unpack(sum_b, a2, a3);
           return (a0 + a1) + (a2 + a3);
         };
-        float hs = exps();
-        if (__any_sync(0xffffffffu, !(hs < kSumLimit))) {
+        // one copy of the exp loop per half, run a second time when the first pass found the maximum stale (the
+        // kernel's instruction footprint decides how often its warps wait for instruction fetches)
+        float hs = 0.f;
+#pragma unroll 1
+        for (int attempt = 0; attempt < 2; ++attempt) {
+          hs = exps();
+          if (attempt == 1 || !__any_sync(0xffffffffu, !(hs < kSumLimit))) break;
           float mxa[4];
 #pragma unroll
           for (int u = 0; u < 4; ++u) mxa[u] = -INFINITY;
@@ -477,7 +482,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
                                    : mbar_wait(smem_u32(&bar_pv0), j & 1, status, kWaitOReady);
             if (ok) {
               tc_fence_after_sync();
-#pragma unroll
+#pragma unroll 1
               for (int c0 = 0; c0 < 128; c0 += 32) {
                 uint32_t r[32];
                 tmem_ld32(tmem_o + lane_off + c0, r);
@@ -488,7 +493,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
               }
             }
           }
-          hs = exps();
         }
         l_sum += hs;
         tmem_st32(tmem_s + lane_off + half * 32, pk);
