@@ -624,6 +624,16 @@ static rbs_status prefill_impl(const rbs_shape* shape, int q_start_block, int n_
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   p.R = x.B / 128;
   if (x.B >= 128) return launch_prefill_tc(p, Q, K, V, x.Hkv, s);   // tensor-core path (blocks of 128 or 256)
+  if (mask == nullptr && (q_start_block & 1) == 0) {
+    // Dense attention does not depend on the block size: blocks of 64 run on the tensor-core path as blocks of 128
+    // (a chunk has to start on a 128-token boundary for that).
+    p.R = 1;
+    p.q0 = q_start_block / 2;
+    p.Mq = (n_q_tokens + 127) / 128;
+    p.M = (x.N + 127) / 128;
+    p.W = (p.M + 31) / 32;
+    return launch_prefill_tc(p, Q, K, V, x.Hkv, s);
+  }
   return launch_prefill<64>(p, s);                                    // blocks of 64: register-softmax mma.sync path
 }
 

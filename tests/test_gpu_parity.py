@@ -364,7 +364,13 @@ def test_chunked_calls_reproduce_the_whole_sequence(B, Mtot, cuts):
         kept += float(dc[0, 0]) * pairs
         oc, lc = rbs_sparse_prefill_chunk(Qc, Kg, Vg, mc, B, q0, return_lse=True)
         assert torch.equal(oc, O[:, t0:t1]) and torch.equal(lc, lse[:, :, t0:t1])
-        assert torch.equal(rbs_sparse_prefill_chunk(Qc, Kg, Vg, None, B, q0), Od[:, t0:t1])
+        od = rbs_sparse_prefill_chunk(Qc, Kg, Vg, None, B, q0)
+        if B == 64 and q0 % 2 == 1:
+            # dense attention with blocks of 64 runs on the 128-row tensor-core kernel when the chunk starts on a
+            # 128-token boundary and on the 64-row kernel otherwise: same values to rounding, not the same bits
+            assert (od.float() - Od[:, t0:t1].float()).abs().max().item() <= OUT_MAX_ABS
+        else:
+            assert torch.equal(od, Od[:, t0:t1])
     assert abs(kept / (cfg.M * (cfg.M + 1) / 2) - float(dens[0, 0])) < 1e-6
 
 
