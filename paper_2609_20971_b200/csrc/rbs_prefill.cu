@@ -584,6 +584,356 @@ static rbs_status launch_prefill_tc(const PrefillParams& p, const rbs_tensor& Q,
   return RBS_OK;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Tensor-core path for blocks of 64.  A 128-row tile holds two consecutive query blocks (rows 0-63: block iA,
+// rows 64-127: block iB = iA + 1), each with its own mask row; the tile walks the union of the two rows in key
+// blocks of 64 and every row half takes part only in the key blocks its own mask row selects (for the other half
+// P is zero and no exponential is computed: the halves are whole warps).  Per key block:
+//   S[128 q x 64 keys] = Q K_b^T   (8 MMAs of K = 16, N = 64)      O[128 q x 128 d] += P V_b   (4 MMAs, K = 64 keys)
+// The work executed is the union of the two rows, so the kernel pays off when neighbouring query blocks select
+// similar key blocks (forced blocks always do).  K and V are double-buffered (16 KB stages): with key blocks this
+// short the next block must already be on its way while the current one is multiplied.
+// TMEM columns: [0,64) S with P (bf16 pairs) over [0,32); [128,256) O.  Roles and CTA shape as in prefill_tc_kernel.
+// ---------------------------------------------------------------------------------------------
+struct Pair64 {
+  const uint32_t* rowA; const uint32_t* rowB;   // mask rows of the two query blocks (rowB null: no second block)
+  int iA, iB;
+  // next key block after `cur` (-1 to start) selected by either row within its causal range, or -1
+  __device__ __forceinline__ int next(int cur) const {
+    const int last = rowB ? iB : iA;
+    int b = cur + 1;
+    while (b <= last) {
+      const int w = b >> 5;
+      uint32_t u = __ldg(rowA + w);
+      if (((w + 1) << 5) - 1 > iA) u = (w << 5) > iA ? 0u : (u & (0xffffffffu >> (31 - (iA & 31))));
+      if (rowB) {
+        uint32_t v = __ldg(rowB + w);
+        if (((w + 1) << 5) - 1 > iB) v = (w << 5) > iB ? 0u : (v & (0xffffffffu >> (31 - (iB & 31))));
+        u |= v;
+      }
+      u >>= (b & 31);
+      if (u) return b + __ffs(u) - 1;
+      b = (b | 31) + 1;
+    }
+    return -1;
+  }
+  // bit 0 / 1: the block is selected by row A / B; bit 2 / 3: it is the diagonal block of row A / B
+  __device__ __forceinline__ uint32_t flags(int b) const {
+    uint32_t f = 0;
+    if (b <= iA && ((__ldg(rowA + (b >> 5)) >> (b & 31)) & 1u)) f |= 1u;
+    if (rowB && b <= iB && ((__ldg(rowB + (b >> 5)) >> (b & 31)) & 1u)) f |= 2u;
+    if (b == iA) f |= 4u;
+    if (b == iB) f |= 8u;
+    return f;
+  }
+};
+
+__global__ void __launch_bounds__(kPfThreads, 2)
+prefill_tc64_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                    const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
+                    const PrefillParams p, unsigned int* status) {
+  constexpr int B = 64;
+  constexpr uint32_t kPanel = 128 * 128;       // Q: 128 rows x 64 bf16 columns = 16 KB
+  constexpr uint32_t kTile = 2 * kPanel;
+  constexpr uint32_t kHalfPanel = 64 * 128;    // K/V: 64 rows x 64 bf16 columns = 8 KB
+  constexpr uint32_t kStage = 2 * kHalfPanel;  // one K or V stage: 16 KB
+  constexpr uint32_t kIdescQK = idesc_bf16_f32(128, 64, false);
+  constexpr uint32_t kIdescPV = idesc_bf16_f32(128, 128, true);
+  extern __shared__ __align__(1024) unsigned char smem[];
+  unsigned char* sQ = smem;
+  unsigned char* sK = smem + kTile;                // two stages
+  unsigned char* sV = smem + kTile + 2 * kStage;   // two stages
+  __shared__ __align__(8) uint64_t bar_q, bar_kfull[2], bar_vfull[2], bar_kempty[2], bar_vempty[2], bar_s, bar_p, bar_pv;
+  __shared__ uint32_t s_tmem;
+  __shared__ uint32_t s_blk[2];   // flags of the key block (see Pair64::flags), bit 4: the tile's last block
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  // tile order as in prefill_tc_kernel, in units of 128-row tiles (two query blocks)
+  const int n_rows = (p.Mq + 1) / 2;
+  const int Hkv = p.Hq / p.G;
+  const int per_band_kv = p.band_rows * p.G;
+  const int per_band = p.L * Hkv * per_band_kv;
+  const int band = static_cast<int>(blockIdx.x / per_band), rem_band = static_cast<int>(blockIdx.x % per_band);
+  const int kvid = rem_band / per_band_kv, rem = rem_band % per_band_kv;
+  const int l = kvid / Hkv, hk = kvid % Hkv;
+  const int Tl = n_rows - 1 - (band * p.band_rows + rem / p.G);   // 128-row tile inside this call's chunk
+  if (Tl < 0) return;
+  const int h = hk * p.G + rem % p.G;
+  Pair64 pr;
+  pr.iA = p.q0 + 2 * Tl;
+  pr.iB = pr.iA + 1;
+  pr.rowA = p.mask + ((static_cast<int64_t>(l) * p.Hq + h) * p.Mq + 2 * Tl) * p.W;
+  pr.rowB = (2 * Tl + 1 < p.Mq) ? pr.rowA + p.W : nullptr;
+
+  if (tid == 0) {
+    mbar_init(smem_u32(&bar_q), 1);
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(smem_u32(&bar_kfull[s]), 1);
+      mbar_init(smem_u32(&bar_vfull[s]), 1);
+      mbar_init(smem_u32(&bar_kempty[s]), 1);
+      mbar_init(smem_u32(&bar_vempty[s]), 1);
+    }
+    mbar_init(smem_u32(&bar_s), 1);
+    mbar_init(smem_u32(&bar_p), 128);
+    mbar_init(smem_u32(&bar_pv), 1);
+    mbar_fence_init();
+  }
+  if (warp == 5) tmem_alloc(smem_u32(&s_tmem), 256);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_s = s_tmem, tmem_o = s_tmem + 128;
+
+  if (warp >= 4) reg_dealloc<48>();
+  if (warp >= 6) {
+    // idle: registers donated above
+  } else if (warp == 4) {
+    // ------------------------------- TMA producer -------------------------------
+    if (lane == 0) {
+      tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
+      int b = pr.next(-1);
+      if (b >= 0) {
+        mbar_arrive_expect_tx(smem_u32(&bar_q), kTile);
+        tma_load_4d(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, Tl * 128, l);
+        tma_load_4d(smem_u32(sQ + kPanel), &tmQ, smem_u32(&bar_q), 64, h, Tl * 128, l);
+      }
+      for (int n = 0; b >= 0; ++n, b = pr.next(b)) {
+        const int st = n & 1;
+        const uint32_t par = ((n >> 1) - 1) & 1;   // the stage's previous use
+        if (n >= 2 && !mbar_wait(smem_u32(&bar_kempty[st]), par, status, kWaitStageFree)) break;
+        mbar_arrive_expect_tx(smem_u32(&bar_kfull[st]), kStage);
+        tma_load_4d(smem_u32(sK + st * kStage), &tmK, smem_u32(&bar_kfull[st]), 0, hk, b * B, l);
+        tma_load_4d(smem_u32(sK + st * kStage + kHalfPanel), &tmK, smem_u32(&bar_kfull[st]), 64, hk, b * B, l);
+        if (n >= 2 && !mbar_wait(smem_u32(&bar_vempty[st]), par, status, kWaitStageFree)) break;
+        mbar_arrive_expect_tx(smem_u32(&bar_vfull[st]), kStage);
+        tma_load_4d(smem_u32(sV + st * kStage), &tmV, smem_u32(&bar_vfull[st]), 0, hk, b * B, l);
+        tma_load_4d(smem_u32(sV + st * kStage + kHalfPanel), &tmV, smem_u32(&bar_vfull[st]), 64, hk, b * B, l);
+      }
+    }
+  } else if (warp == 5) {
+    // ------------------------------- MMA issuer -------------------------------
+    // The whole warp runs this loop in lock step and one elected lane issues each tcgen05 instruction.
+    int b = pr.next(-1);
+    bool ok = b < 0 || mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
+    ok = __all_sync(0xffffffffu, ok);
+    const uint64_t dq = smem_desc_sw128(smem_u32(sQ), 16, 1024);
+    uint64_t dk[2], dv[2];
+#pragma unroll
+    for (int s = 0; s < 2; ++s) {
+      dk[s] = smem_desc_sw128(smem_u32(sK + s * kStage), 16, 1024);
+      dv[s] = smem_desc_sw128(smem_u32(sV + s * kStage), kHalfPanel, 1024);
+    }
+    int b_next = b >= 0 ? pr.next(b) : -1;
+    auto issue_qk = [&](int n, int blk, int blk_next) {
+      if (lane == 0) {
+        s_blk[n & 1] = pr.flags(blk) | (blk_next < 0 ? 16u : 0u);
+        __threadfence_block();
+      }
+      __syncwarp();
+      const int st = n & 1;
+      mma_ss_k128_commit_elect(tmem_s, dq, st ? dk[1] : dk[0], kIdescQK, kPanel, kHalfPanel, smem_u32(&bar_kempty[st]));
+      mma_commit_elect(smem_u32(&bar_s));
+    };
+    if (ok && b >= 0) {
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull[0]), 0, status, kWaitTmaFull));
+      if (ok) {
+        tc_fence_after_sync();
+        issue_qk(0, b, b_next);
+      }
+    }
+    for (int n = 0; ok && b >= 0; ++n) {
+      const int st = n & 1;
+      const uint32_t ph = n & 1, sph = (n >> 1) & 1;
+      const int b_next2 = b_next >= 0 ? pr.next(b_next) : -1;   // global-memory latency hidden behind the softmax
+      // K of the next block is checked before the wait for P: the check stays off the tile's critical path
+      if (b_next >= 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull[st ^ 1]), ((n + 1) >> 1) & 1, status, kWaitTmaFull));
+      ok = ok && __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_vfull[st]), sph, status, kWaitTmaFull) &&
+                                             mbar_wait(smem_u32(&bar_p), ph, status, kWaitPReady));
+      if (!ok) break;
+      tc_fence_after_sync();
+      mma_ts_k64_elect(tmem_o, tmem_s, st ? dv[1] : dv[0], kIdescPV, 2048 >> 4, n != 0, smem_u32(&bar_vempty[st]));
+      mma_commit_elect(smem_u32(&bar_pv));
+      if (b_next >= 0) issue_qk(n + 1, b_next, b_next2);
+      b = b_next;
+      b_next = b_next2;
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------- softmax: one query row per thread -------------------------------
+    reg_alloc<208>();
+    const int row = warp * 32 + lane;
+    const int rh = warp >> 1;                       // row half: 0 = block iA, 1 = block iB (whole warps)
+    const int rloc = row - rh * 64;                 // row inside its query block
+    const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
+    float m_used = -INFINITY, l_sum = 0.f;          // m_used in log2 units of the scaled logits
+    const bool any_block = pr.next(-1) >= 0;
+    bool ok = true;
+    int n = 0;
+    const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
+    for (bool more = any_block; more; ++n) {
+      if (!(ok = mbar_wait(smem_u32(&bar_s), n & 1, status, kWaitMmaDone))) break;
+      const uint32_t blk = *reinterpret_cast<volatile uint32_t*>(&s_blk[n & 1]);
+      more = (blk & 16u) == 0u;
+      tc_fence_after_sync();
+      uint32_t pk[32];
+      if ((blk >> rh) & 1u) {   // this row half attends the block
+        uint32_t s[64];
+        {
+          uint32_t(&s0)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[0]);
+          uint32_t(&s1)[32] = *reinterpret_cast<uint32_t(*)[32]>(&s[32]);
+          tmem_ld32(tmem_s + lane_off, s0);
+          tmem_ld32(tmem_s + lane_off + 32, s1);
+          tmem_wait_ld();
+        }
+        if ((blk >> (2 + rh)) & 1u) {   // the half's diagonal block: keys after the query are hidden
+#pragma unroll
+          for (int c = 0; c < 64; ++c)
+            if (c > rloc) s[c] = 0xff800000u;   // -inf
+        }
+        // lazy running maximum, as in prefill_tc_kernel
+        auto exps = [&]() -> float {
+          const uint64_t negm2 = f2_pack(-m_used, -m_used);
+          uint64_t sum_a = 0ull, sum_b = 0ull;   // (0.f, 0.f)
+#pragma unroll
+          for (int q = 0; q < 64; q += 4) {
+            const uint64_t x01 = f2_fma(f2_pack(__uint_as_float(s[q]), __uint_as_float(s[q + 1])), scale2, negm2);
+            const uint64_t x23 = f2_fma(f2_pack(__uint_as_float(s[q + 2]), __uint_as_float(s[q + 3])), scale2, negm2);
+            float x0, x1, x2, x3;
+            f2_unpack(x01, x0, x1);
+            f2_unpack(x23, x2, x3);
+            const float p0 = fast_exp2(x0), p1 = fast_exp2(x1), p2 = fast_exp2(x2), p3 = fast_exp2(x3);
+            sum_a = f2_add(sum_a, f2_pack(p0, p1));
+            sum_b = f2_add(sum_b, f2_pack(p2, p3));
+            pk[q >> 1] = pack_bf16(p0, p1);
+            pk[(q >> 1) + 1] = pack_bf16(p2, p3);
+          }
+          float a0, a1, a2, a3;
+          f2_unpack(sum_a, a0, a1);
+          f2_unpack(sum_b, a2, a3);
+          return (a0 + a1) + (a2 + a3);
+        };
+        float hs = 0.f;
+#pragma unroll 1
+        for (int attempt = 0; attempt < 2; ++attempt) {
+          hs = exps();
+          if (attempt == 1 || !__any_sync(0xffffffffu, !(hs < kSumLimit))) break;
+          float mxa[4];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) mxa[u] = -INFINITY;
+#pragma unroll
+          for (int c = 0; c < 64; c += 8) {
+#pragma unroll
+            for (int u = 0; u < 4; ++u) mxa[u] = max3(mxa[u], __uint_as_float(s[c + 2 * u]), __uint_as_float(s[c + 2 * u + 1]));
+          }
+          const float mx = fmaxf(fmaxf(mxa[0], mxa[1]), fmaxf(mxa[2], mxa[3])) * p.scale_log2;
+          const float m_new = fmaxf(m_used, mx);
+          const float corr = fast_exp2(m_used - m_new);     // 0 while m_used = -inf
+          l_sum *= corr;
+          m_used = m_new;
+          if (n > 0) {   // O holds the P V of everything issued so far: wait for it, then rescale
+            if (ok) ok = mbar_wait(smem_u32(&bar_pv), (n - 1) & 1, status, kWaitOReady);
+            if (ok) {
+              tc_fence_after_sync();
+#pragma unroll 1
+              for (int c0 = 0; c0 < 128; c0 += 32) {
+                uint32_t r[32];
+                tmem_ld32(tmem_o + lane_off + c0, r);
+                tmem_wait_ld();
+#pragma unroll
+                for (int q = 0; q < 32; ++q) r[q] = __float_as_uint(__uint_as_float(r[q]) * corr);
+                tmem_st32(tmem_o + lane_off + c0, r);
+              }
+            }
+          }
+        }
+        l_sum += hs;
+      } else {
+#pragma unroll
+        for (int q = 0; q < 32; ++q) pk[q] = 0u;   // P = 0 for the rows whose block did not select these keys
+      }
+      tmem_st32(tmem_s + lane_off, pk);
+      tmem_wait_st();
+      tc_fence_before_sync();
+      mbar_arrive(smem_u32(&bar_p));
+      if (!ok) break;
+    }
+    // epilogue: O / l -> bf16 -> global
+    const int64_t tok = static_cast<int64_t>(Tl) * 128 + row;
+    __nv_bfloat16* orow = p.O + l * p.osb + tok * p.ost + h * p.osh;
+    float* lse_dst = p.lse ? p.lse + (static_cast<int64_t>(l) * p.Hq + h) * p.Nq + tok : nullptr;
+    const bool in_seq = tok < p.Nq;   // rows past the end of the queries are not written
+    if (!any_block) {
+      if (in_seq) {
+#pragma unroll
+        for (int c = 0; c < 16; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
+        if (lse_dst) *lse_dst = -INFINITY;
+      }
+    } else {
+      // every thread of the four warps reaches the barrier below, also one whose wait has given up
+      const bool o_ready = __all_sync(0xffffffffu, ok && mbar_wait(smem_u32(&bar_pv), (n - 1) & 1, status, kWaitOReady));
+      tc_fence_after_sync();
+      const bool empty_row = !(l_sum > 0.f);          // a row whose own block selected nothing: zeros, lse = -inf
+      const float inv = empty_row ? 0.f : 1.0f / l_sum;
+      const uint32_t srow = smem_u32(sQ) + row * 128;
+#pragma unroll
+      for (int c0 = 0; o_ready && c0 < 128; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem_o + lane_off + c0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int q = 0; q < 32; q += 8) {
+          uint4 v;
+          v.x = pack_bf16(__uint_as_float(r[q]) * inv, __uint_as_float(r[q + 1]) * inv);
+          v.y = pack_bf16(__uint_as_float(r[q + 2]) * inv, __uint_as_float(r[q + 3]) * inv);
+          v.z = pack_bf16(__uint_as_float(r[q + 4]) * inv, __uint_as_float(r[q + 5]) * inv);
+          v.w = pack_bf16(__uint_as_float(r[q + 6]) * inv, __uint_as_float(r[q + 7]) * inv);
+          if (empty_row) v = make_uint4(0, 0, 0, 0);
+          const int chunk = (c0 + q) >> 3;   // 16-byte piece 0..15 of the row
+          const uint32_t dst = srow + (chunk >> 3) * kPanel + (((chunk & 7) ^ (row & 7)) << 4);
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+        }
+      }
+      fence_proxy_async_smem();
+      asm volatile("bar.sync 1, 128;" ::: "memory");   // the four softmax warps
+      if (tid == 0 && o_ready) {
+        tma_store_4d(&tmO, smem_u32(sQ), 0, h, Tl * 128, l);
+        tma_store_4d(&tmO, smem_u32(sQ + kPanel), 64, h, Tl * 128, l);
+        tma_store_commit();
+        tma_store_wait_read();
+      }
+      if (lse_dst && in_seq && o_ready) *lse_dst = empty_row ? -INFINITY : (m_used + fast_log2(l_sum)) * 0.6931471805599453f;
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  if (warp == 5) tmem_dealloc(s_tmem, 256);
+}
+
+static rbs_status launch_prefill_tc64(const PrefillParams& p, const rbs_tensor& Q, const rbs_tensor& K,
+                                      const rbs_tensor& V, int Hkv, cudaStream_t s) {
+  CUtensorMap tmQ, tmK, tmV, tmO;
+  rbs_status st;
+  if ((st = make_tmap_lthd(&tmQ, Q.ptr, p.L, p.Nq, p.Hq, kHeadDim, Q.stride_batch, Q.stride_token, Q.stride_head, 64, 128, true)) != RBS_OK) return st;
+  if ((st = make_tmap_lthd(&tmK, K.ptr, p.L, p.N, Hkv, kHeadDim, K.stride_batch, K.stride_token, K.stride_head, 64, 64, true)) != RBS_OK) return st;
+  if ((st = make_tmap_lthd(&tmV, V.ptr, p.L, p.N, Hkv, kHeadDim, V.stride_batch, V.stride_token, V.stride_head, 64, 64, true)) != RBS_OK) return st;
+  if ((st = make_tmap_lthd(&tmO, p.O, p.L, p.Nq, p.Hq, kHeadDim, p.osb, p.ost, p.osh, 64, 128, true)) != RBS_OK) return st;
+  unsigned int* status = device_status_ptr();
+  if (status == nullptr) return RBS_ERR_CUDA;
+  const size_t smem = 2 * 128 * 128 + 4 * 2 * 64 * 128;   // Q + two stages each of K and V
+  RBS_CUDA_OK(cudaFuncSetAttribute(prefill_tc64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  PrefillParams pp = p;
+  const int n_rows = (p.Mq + 1) / 2;
+  int n_bands = n_rows / 64;
+  n_bands = n_bands < 1 ? 1 : (n_bands > 4 ? 4 : n_bands);
+  pp.band_rows = (n_rows + n_bands - 1) / n_bands;
+  const long long n_cta = static_cast<long long>(p.L) * p.Hq * pp.band_rows * n_bands;
+  if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
+  prefill_tc64_kernel<<<static_cast<unsigned>(n_cta), kPfThreads, smem, s>>>(tmQ, tmK, tmV, tmO, pp, status);
+  RBS_CUDA_OK(cudaGetLastError());
+  return RBS_OK;
+}
+
 template <int B>
 static rbs_status launch_prefill(const PrefillParams& p, cudaStream_t s) {
   const size_t smem = static_cast<size_t>(5) * B * 256;
@@ -634,7 +984,8 @@ static rbs_status prefill_impl(const rbs_shape* shape, int q_start_block, int n_
     p.W = (p.M + 31) / 32;
     return launch_prefill_tc(p, Q, K, V, x.Hkv, s);
   }
-  return launch_prefill<64>(p, s);                                    // blocks of 64: register-softmax mma.sync path
+  if (mask != nullptr) return launch_prefill_tc64(p, Q, K, V, x.Hkv, s);   // blocks of 64, two query blocks per tile
+  return launch_prefill<64>(p, s);   // dense chunk from an odd block of 64: register-softmax mma.sync kernel
 }
 
 extern "C" rbs_status rbs_sparse_prefill(const rbs_shape* shape, rbs_tensor Q, rbs_tensor K, rbs_tensor V,
