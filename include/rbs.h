@@ -186,7 +186,9 @@ RBS_API rbs_status rbs_select_variant(const rbs_shape* shape, rbs_tensor Q, rbs_
  * e.g. one 128K-token layer with 4 KV heads at block 128 needs about half of it).
  * The call itself performs no cudaMalloc / cudaFree and calls no allocating library routine.
  * The first call on each device looks up the array's device address (and, like any first use of a CUDA
- * module, lets the driver load the kernels); make that first call outside stream capture.
+ * module, lets the driver load the kernels, which is also when the driver places the array in device memory);
+ * make that first call outside stream capture and before the application claims the rest of the device's memory --
+ * a caller that has already taken every free byte gets RBS_ERR_CUDA from it.
  * All calls on one device share the one array: it keeps whatever the previous call left there, the
  * parts that must start at zero are cleared by every call, and two calls whose kernels may overlap on
  * the GPU (different streams without an ordering between them) race on it -- order them.

@@ -73,6 +73,10 @@ def load_library() -> ctypes.CDLL:
                                        vp, f, vp, sz, vp]
     lib.rbs_device_status.restype = i
     lib.rbs_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint), i]
+    lib.rbs_selftest_device_table.restype = i
+    lib.rbs_selftest_device_table.argtypes = []
+    lib.rbs_selftest_wait_timeout.restype = i
+    lib.rbs_selftest_wait_timeout.argtypes = [ctypes.c_uint, vp, vp]
     lib.rbs_status_string.restype = ctypes.c_char_p
     lib.rbs_status_string.argtypes = [i]
     lib.rbs_version.restype = ctypes.c_char_p
@@ -139,6 +143,14 @@ def rbs_device_status(clear: bool = True) -> int:
     if rc not in (0, 5):
         _check(rc, "rbs_device_status")
     return int(code.value)
+
+
+def rbs_selftest_wait_timeout(spin_limit: int = 4096) -> torch.Tensor:
+    """Launches the library's time-out self-test (one thread waits, with a short limit, on a barrier nothing arrives
+    on) and returns the device flag it writes (1 = the wait gave up).  The status word then holds the code."""
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    _check(load_library().rbs_selftest_wait_timeout(spin_limit, _ptr(flag), _stream()), "rbs_selftest_wait_timeout")
+    return flag
 
 
 def rbs_block_stats(K: torch.Tensor, block: int, stats: BlockStats | None = None) -> BlockStats:

@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "rbs.h"
 
 struct CUtensorMap_st;
@@ -49,9 +51,39 @@ SelectWorkspace select_workspace(const Dims& x);
 rbs_status make_tmap_lthd(::CUtensorMap_st* out, const void* ptr, int L, int N, int H, int d, int64_t sb, int64_t st,
                           int64_t sh, int box_d, int box_t, bool swizzle128);
 rbs_status make_tmap_2d(::CUtensorMap_st* out, const void* ptr, int64_t rows, int cols, int box_cols, int box_rows);
+// Number of SMs of the current device (looked up once per device).
 int sm_count();
-// Device address of the status word that bounded waits report to (nullptr if it cannot be obtained).
+// Device address, on the current device, of the status word that bounded waits report to (nullptr if it cannot be
+// obtained).  Looked up once per device, with that device current: an address taken on one GPU means nothing on another.
 unsigned int* device_status_ptr();
+// cudaFuncSetAttribute(MaxDynamicSharedMemorySize) only when this (kernel, device) has not yet been given at least
+// `bytes`: the attribute is per device and sticky, and the call is not free on the per-layer path.
+rbs_status ensure_dynamic_smem(const void* kernel, size_t bytes);
+
+// A value per CUDA device, filled on first use by `make(device, &value)` (true = success; failures are not cached).
+// The table itself is plain host logic: it never touches CUDA, so it is also exercised without a GPU.
+template <typename T, int kMaxDevices = 64>
+class PerDevice {
+ public:
+  template <typename Make>
+  bool get(int device, T* out, Make make) {
+    if (device < 0 || device >= kMaxDevices) return false;
+    std::lock_guard<std::mutex> guard(lock_);
+    if (!have_[device]) {
+      T v{};
+      if (!make(device, &v)) return false;
+      value_[device] = v;
+      have_[device] = true;
+    }
+    *out = value_[device];
+    return true;
+  }
+
+ private:
+  std::mutex lock_;
+  bool have_[kMaxDevices] = {};
+  T value_[kMaxDevices] = {};
+};
 
 #define RBS_CUDA_OK(expr)                               \
   do {                                                  \

@@ -1,6 +1,9 @@
 // rbs_sparse_prefill: causal block-sparse attention over a bit-packed block mask (Sec. 3.3), dense when
-// the mask is NULL (Eq. 1).  One CTA per (batch, query head, query block); it walks the set bits of its
-// mask row, streams those K/V blocks through shared memory and keeps an online softmax in registers.
+// the mask is NULL (Eq. 1).  The work horses are the tcgen05 kernels further down (prefill_tc_kernel for blocks of
+// 128 and 256, prefill_tc64_kernel for blocks of 64): TMA-fed K/V tiles, S and O accumulators in tensor memory,
+// one softmax thread per query row with a lazily updated running maximum, the key list walked straight from the
+// mask bits.  prefill_mma_kernel (mma.sync, softmax in registers) only serves a dense chunk that starts on an odd
+// block of 64.
 #include "rbs_common.cuh"
 #include "rbs_sm100.cuh"
 
@@ -568,7 +571,7 @@ static rbs_status launch_prefill_tc(const PrefillParams& p, const rbs_tensor& Q,
   unsigned int* status = device_status_ptr();
   if (status == nullptr) return RBS_ERR_CUDA;
   const size_t smem = 3 * 2 * 128 * 128;
-  RBS_CUDA_OK(cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  if ((st = ensure_dynamic_smem(reinterpret_cast<const void*>(prefill_tc_kernel), smem)) != RBS_OK) return st;
   PrefillParams pp = p;
   const int n_rows = p.Mq * p.R;
   // up to four bands of at least 64 query tiles (512 CTAs per band and KV head at G = 8: enough to fill the GPU
@@ -921,7 +924,7 @@ static rbs_status launch_prefill_tc64(const PrefillParams& p, const rbs_tensor& 
   unsigned int* status = device_status_ptr();
   if (status == nullptr) return RBS_ERR_CUDA;
   const size_t smem = 2 * 128 * 128 + 4 * 2 * 64 * 128;   // Q + two stages each of K and V
-  RBS_CUDA_OK(cudaFuncSetAttribute(prefill_tc64_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  if ((st = ensure_dynamic_smem(reinterpret_cast<const void*>(prefill_tc64_kernel), smem)) != RBS_OK) return st;
   PrefillParams pp = p;
   const int n_rows = (p.Mq + 1) / 2;
   int n_bands = n_rows / 64;
@@ -937,7 +940,7 @@ static rbs_status launch_prefill_tc64(const PrefillParams& p, const rbs_tensor& 
 template <int B>
 static rbs_status launch_prefill(const PrefillParams& p, cudaStream_t s) {
   const size_t smem = static_cast<size_t>(5) * B * 256;
-  RBS_CUDA_OK(cudaFuncSetAttribute(prefill_mma_kernel<B>, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  { const rbs_status st = ensure_dynamic_smem(reinterpret_cast<const void*>(prefill_mma_kernel<B>), smem); if (st != RBS_OK) return st; }
   const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.Mq;
   if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
   prefill_mma_kernel<B><<<static_cast<unsigned>(n_cta), B * 2, smem, s>>>(p);

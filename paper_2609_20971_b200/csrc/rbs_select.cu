@@ -387,7 +387,7 @@ static rbs_status launch_select_tc(const SelectParams& p, const rbs_tensor& Q, c
   const size_t smem = static_cast<size_t>(4) * 128 * 128 + 2 * static_cast<size_t>(B) * 128 +
                       (B + 32) * sizeof(float) + 2 * static_cast<size_t>(n_tiles_max) * 128 * sizeof(float);
   auto kern = select_tc_kernel<B>;
-  RBS_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  if ((st = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem)) != RBS_OK) return st;
   const long long n_cta = static_cast<long long>(p.L) * p.Hq * p.Mq;
   if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
   kern<<<static_cast<unsigned>(n_cta), kTcThreads, smem, s>>>(tmQ, tmChi, tmClo, p, status);

@@ -14,6 +14,7 @@ namespace rbs {
 
 enum : unsigned int {
   kWaitTmaFull = 1, kWaitStageFree = 2, kWaitMmaDone = 3, kWaitTmemFree = 4, kWaitPReady = 5, kWaitOReady = 6,
+  kWaitSelfTest = 7,
 };
 
 // ------------------------------------------------------------------------------------------- mbarrier
@@ -41,8 +42,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Waits for the phase with the given parity to complete.  Bounded: after kSpinLimit failed probes the
 // wait gives up, records `code` in the device status word and returns false; callers then drain and exit.
 constexpr uint32_t kSpinLimit = 1u << 24;
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned int* status, unsigned int code) {
-  for (uint32_t it = 0; it < kSpinLimit; ++it) {
+__device__ __forceinline__ bool mbar_wait_limit(uint32_t bar, uint32_t parity, unsigned int* status, unsigned int code,
+                                                uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (it > 2048) __nanosleep(64);
     // once any wait anywhere has given up, the launch is lost: stop waiting everywhere
@@ -50,6 +52,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigne
   }
   atomicCAS(status, 0u, code);
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigned int* status, unsigned int code) {
+  return mbar_wait_limit(bar, parity, status, code, kSpinLimit);
 }
 
 // ------------------------------------------------------------------------------------------- TMA

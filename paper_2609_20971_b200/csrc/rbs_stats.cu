@@ -167,7 +167,7 @@ static rbs_status launch_stats_warp(const rbs_tensor& K, const Dims& x, const rb
   if (status == nullptr) return RBS_ERR_CUDA;
   const size_t smem = static_cast<size_t>(NW) * NS * (B / WPB) * 256;
   auto kern = block_stats_warp_kernel<B, NW, NS, WPB>;
-  RBS_CUDA_OK(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)));
+  if ((st = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem)) != RBS_OK) return st;
   const long long n_tiles = static_cast<long long>(x.L) * x.Hkv * x.M;
   long long want = (n_tiles + NW / WPB - 1) / (NW / WPB);
   const int grid = static_cast<int>(want < sm_count() ? want : sm_count());

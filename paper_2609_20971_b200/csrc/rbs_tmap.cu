@@ -2,19 +2,26 @@
 // (the library does not link against the driver library, so it loads on machines without one).
 #include "rbs_common.cuh"
 #include "rbs_sm100.cuh"
+#include "rbs_selftest.h"
 
 namespace rbs {
 
 static __device__ unsigned int g_device_status = 0;
 
+static bool current_device(int* dev) { return cudaGetDevice(dev) == cudaSuccess; }
+
 unsigned int* device_status_ptr() {
-  static unsigned int* p = nullptr;
-  if (p == nullptr) {
-    void* q = nullptr;
-    if (cudaGetSymbolAddress(&q, g_device_status) != cudaSuccess) return nullptr;
-    p = static_cast<unsigned int*>(q);
-  }
-  return p;
+  static PerDevice<unsigned int*> table;
+  int dev = -1;
+  if (!current_device(&dev)) return nullptr;
+  unsigned int* p = nullptr;
+  const bool ok = table.get(dev, &p, [](int, unsigned int** out) {
+    void* q = nullptr;   // the symbol's address on the device that is current now
+    if (cudaGetSymbolAddress(&q, g_device_status) != cudaSuccess || q == nullptr) return false;
+    *out = static_cast<unsigned int*>(q);
+    return true;
+  });
+  return ok ? p : nullptr;
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -68,13 +75,40 @@ rbs_status make_tmap_2d(CUtensorMap* out, const void* ptr, int64_t rows, int col
 }
 
 int sm_count() {
-  static int n = 0;
-  if (n == 0) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
-  }
-  return n;
+  static PerDevice<int> table;
+  int dev = -1, n = 0;
+  if (!current_device(&dev)) return 148;
+  const bool ok = table.get(dev, &n, [](int d, int* out) {
+    return cudaDeviceGetAttribute(out, cudaDevAttrMultiProcessorCount, d) == cudaSuccess && *out > 0;
+  });
+  return ok ? n : 148;
+}
+
+rbs_status ensure_dynamic_smem(const void* kernel, size_t bytes) {
+  struct Key { const void* fn; int dev; size_t bytes; };
+  static std::mutex lock;
+  static Key seen[256];
+  static int n_seen = 0;
+  int dev = -1;
+  if (!current_device(&dev)) return RBS_ERR_CUDA;
+  std::lock_guard<std::mutex> guard(lock);
+  Key* slot = nullptr;
+  for (int k = 0; k < n_seen; ++k)
+    if (seen[k].fn == kernel && seen[k].dev == dev) { slot = &seen[k]; break; }
+  if (slot != nullptr && slot->bytes >= bytes) return RBS_OK;
+  RBS_CUDA_OK(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(bytes)));
+  if (slot == nullptr && n_seen < 256) slot = &seen[n_seen++];
+  if (slot != nullptr) { slot->fn = kernel; slot->dev = dev; slot->bytes = bytes; }
+  return RBS_OK;
+}
+
+// One CTA, one thread: waits on an mbarrier that nothing ever arrives on, with the given probe limit.
+__global__ void selftest_wait_kernel(unsigned int* status, unsigned int spin_limit, unsigned int* gave_up) {
+  __shared__ __align__(8) uint64_t bar;
+  mbar_init(smem_u32(&bar), 1);
+  mbar_fence_init();
+  const bool ok = mbar_wait_limit(smem_u32(&bar), 0, status, kWaitSelfTest, spin_limit);
+  *gave_up = ok ? 0u : 1u;
 }
 
 }  // namespace rbs
@@ -90,4 +124,40 @@ extern "C" rbs_status rbs_device_status(void* stream, unsigned int* code_out, in
   }
   if (code_out) *code_out = code;
   return code == 0 ? RBS_OK : RBS_ERR_TIMEOUT;
+}
+
+// ---------------------------------------------------------------------------------------------
+// self-tests (include/rbs_selftest.h)
+// ---------------------------------------------------------------------------------------------
+extern "C" int rbs_selftest_device_table(void) {
+  // the per-device table with a fake lookup: every device gets its own value, looked up exactly once; a failed
+  // lookup is not remembered; out-of-range devices are refused
+  rbs::PerDevice<long, 8> table;
+  int calls[8] = {0};
+  bool fail_next = true;
+  auto make = [&](int dev, long* out) {
+    ++calls[dev];
+    if (dev == 5 && fail_next) { fail_next = false; return false; }
+    *out = 1000 + 7 * dev;
+    return true;
+  };
+  long v = 0;
+  const int order[] = {3, 0, 3, 7, 0, 3};
+  for (int dev : order) {
+    if (!table.get(dev, &v, make) || v != 1000 + 7 * dev) return 1;
+  }
+  if (calls[3] != 1 || calls[0] != 1 || calls[7] != 1 || calls[1] != 0) return 2;
+  if (table.get(5, &v, make)) return 3;                 // first lookup fails and must not be cached
+  if (!table.get(5, &v, make) || v != 1035 || calls[5] != 2) return 4;
+  if (table.get(-1, &v, make) || table.get(8, &v, make)) return 5;
+  return 0;
+}
+
+extern "C" rbs_status rbs_selftest_wait_timeout(unsigned int spin_limit, unsigned int* gave_up, void* stream) {
+  if (gave_up == nullptr || spin_limit == 0 || spin_limit > (1u << 16)) return RBS_ERR_INVALID_ARG;
+  unsigned int* status = rbs::device_status_ptr();
+  if (status == nullptr) return RBS_ERR_CUDA;
+  rbs::selftest_wait_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(status, spin_limit, gave_up);
+  RBS_CUDA_OK(cudaGetLastError());
+  return RBS_OK;
 }

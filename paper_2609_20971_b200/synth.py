@@ -75,8 +75,9 @@ def paper_configs() -> dict:
     }
 
 
-def make_inputs(cfg: SynthConfig):
-    """Returns (Q [L,N,Hq,d], K [L,N,Hkv,d], V [L,N,Hkv,d]) as contiguous bf16 CPU tensors."""
+def iter_layers(cfg: SynthConfig):
+    """Yields (l, Q_l [N,Hq,d], K_l [N,Hkv,d], V_l [N,Hkv,d]) as bf16 CPU tensors, one layer of the batch at a
+    time, in order: the same bits make_inputs returns, without holding all layers on the host at once."""
     L, N, Hq, Hkv, d, B = cfg.L, cfg.N, cfg.Hq, cfg.Hkv, cfg.d, cfg.B
     assert Hq % Hkv == 0
     n_keep = N                       # a length that is not a multiple of B is generated padded, then cut
@@ -94,16 +95,13 @@ def make_inputs(cfg: SynthConfig):
     else:
         sigma = torch.full((L, Hkv), float(cfg.sigma))
 
-    Q = torch.empty(L, N, Hq, d, dtype=torch.bfloat16)
-    K = torch.empty(L, N, Hkv, d, dtype=torch.bfloat16)
-    V = torch.empty(L, N, Hkv, d, dtype=torch.bfloat16)
     for l in range(L):
-        V[l] = randn(N, Hkv, d).to(torch.bfloat16)
+        Vl = randn(N, Hkv, d).to(torch.bfloat16)
         muq = randn(M, 1, Hq, d)
         q = randn(M, B, Hq, d)
         if cfg.s_q != 0.0:
             q += cfg.s_q * muq
-        Q[l] = q.view(N, Hq, d).to(torch.bfloat16)
+        Ql = q.view(N, Hq, d).to(torch.bfloat16)
         del q
         mu = randn(M, 1, Hkv, d)
         k = mu + sigma[l].view(1, 1, Hkv, 1) * randn(M, B, Hkv, d)
@@ -119,14 +117,24 @@ def make_inputs(cfg: SynthConfig):
             jj = bb + torch.floor(frac[bb, hh] * (M - bb).float()).long()
             jj = torch.clamp(jj, max=M - 1)
             qh = hh * G + which[bb, hh]
-            qmean = Q[l].view(M, B, Hq, d).float().mean(dim=1)        # [M, Hq, d]
+            qmean = Ql.view(M, B, Hq, d).float().mean(dim=1)          # [M, Hq, d]
             u = qmean[jj, qh]                                         # [n, d]
             u = u / u.norm(dim=1, keepdim=True).clamp_min(1e-12)
             k[bb, pos[bb, hh], hh] = cfg.nu * math.sqrt(d) * u
-        K[l] = k.view(N, Hkv, d).to(torch.bfloat16)
+        Kl = k.view(N, Hkv, d).to(torch.bfloat16)
         del k
-    if n_keep != N:
-        Q, K, V = (t[:, :n_keep].contiguous() for t in (Q, K, V))
+        if n_keep != N:
+            Ql, Kl, Vl = (t[:n_keep].contiguous() for t in (Ql, Kl, Vl))
+        yield l, Ql, Kl, Vl
+
+
+def make_inputs(cfg: SynthConfig):
+    """Returns (Q [L,N,Hq,d], K [L,N,Hkv,d], V [L,N,Hkv,d]) as contiguous bf16 CPU tensors."""
+    Q = torch.empty(cfg.L, cfg.N, cfg.Hq, cfg.d, dtype=torch.bfloat16)
+    K = torch.empty(cfg.L, cfg.N, cfg.Hkv, cfg.d, dtype=torch.bfloat16)
+    V = torch.empty(cfg.L, cfg.N, cfg.Hkv, cfg.d, dtype=torch.bfloat16)
+    for l, Ql, Kl, Vl in iter_layers(cfg):
+        Q[l], K[l], V[l] = Ql, Kl, Vl
     return Q, K, V
 
 

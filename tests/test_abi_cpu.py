@@ -21,13 +21,18 @@ def lib():
 
 
 def declared_functions():
-    text = open(os.path.join(ROOT, "include", "rbs.h")).read()
-    return re.findall(r"RBS_API\s+[\w\s\*]+?\b(rbs_\w+)\s*\(", text)
+    names = []
+    inc = os.path.join(ROOT, "include")
+    for header in sorted(os.listdir(inc)):
+        if header.endswith(".h"):
+            names += re.findall(r"RBS_API\s+[\w\s\*]+?\b(rbs_\w+)\s*\(", open(os.path.join(inc, header)).read())
+    return names
 
 
 def test_every_declared_symbol_is_exported(lib):
     names = declared_functions()
-    assert {"rbs_block_stats", "rbs_select", "rbs_sparse_prefill", "rbs_workspace_bytes"} <= set(names)
+    assert {"rbs_block_stats", "rbs_select", "rbs_sparse_prefill", "rbs_workspace_bytes",
+            "rbs_selftest_device_table", "rbs_selftest_wait_timeout"} <= set(names)
     for n in names:
         assert hasattr(lib, n), n
 
@@ -121,3 +126,16 @@ def test_group_union_argument_checks(lib):
     assert lib.rbs_mask_group_union(ctypes.byref(good), 7, 256, p, p, None) == INVALID      # past the end
     bad = RbsShape(1, 1024, 3, 2, 128, 128)
     assert lib.rbs_mask_group_union(ctypes.byref(bad), 0, -1, p, p, None) == UNSUPPORTED
+
+
+def test_per_device_lookup_table(lib):
+    """Values such as the device address of the status word are looked up once per device and never handed to
+    another device: the table logic is host-only and is checked here with a fake lookup (0 = every check passed)."""
+    assert lib.rbs_selftest_device_table() == 0
+
+
+def test_wait_timeout_selftest_argument_checks(lib):
+    p = ctypes.c_void_p(0x1000)
+    assert lib.rbs_selftest_wait_timeout(0, p, None) == INVALID
+    assert lib.rbs_selftest_wait_timeout(1 << 20, p, None) == INVALID      # only short limits are accepted
+    assert lib.rbs_selftest_wait_timeout(1024, None, None) == INVALID

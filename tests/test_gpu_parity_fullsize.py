@@ -64,6 +64,35 @@ def test_fullsize_stats_and_selection(full):
     assert np.array_equal(full["dens"].cpu().numpy(), (pop / (M * (M + 1) / 2)).astype(np.float32))
 
 
+def test_fullsize_whole_mask(full):
+    """Every row of every head of the 128K mask (32 x 1,024 rows; base, rescue and final) against the selector oracle
+    run in full: identical outside the 1e-3 band around each branch threshold, and the number of differing decisions
+    inside the band stays small."""
+    cfg = full["cfg"]
+    M, B, G = cfg.M, cfg.B, cfg.Hq // cfg.Hkv
+    words = {k: full[k].cpu().numpy().view(np.uint32)[0] for k in ("mask", "mb", "mr")}       # [Hq, M, W]
+
+    def bits(w):   # [M, W] uint32 -> [M, M] bool
+        return np.unpackbits(w.view(np.uint8), axis=1, bitorder="little")[:, :M].astype(bool)
+    n_mismatch = 0
+    for hk in range(cfg.Hkv):
+        c, r = orc.block_stats(to_f64(full["K"][0, :, hk]), B)
+        beta, _, _ = orc.rescue_coefficient(r)
+        for h in range(hk * G, (hk + 1) * G):
+            sel = orc.select_head(to_f64(full["Q"][0, :, h]), c, r, beta, B, cfg.alpha_base, cfg.alpha_rescue,
+                                  cfg.n_sink, cfg.n_local, cfg.n_recent)
+            near_b, near_r = sel.margin_base <= 1e-3, sel.margin_rescue <= 1e-3
+            got, got_b, got_r = bits(words["mask"][h]), bits(words["mb"][h]), bits(words["mr"][h])
+            assert not ((got_b != sel.base) & ~near_b).any(), h
+            assert not ((got_r != sel.rescue) & ~near_r).any(), h
+            assert not ((got != sel.final) & ~(near_b | near_r)).any(), h
+            assert np.array_equal(got, got_b | got_r | sel.forced)      # the union is exact on the GPU's own branches
+            assert not np.triu(got, 1).any()
+            n_mismatch += int((got != sel.final).sum())
+            assert abs(float(full["dens"][0, h]) - sel.density) <= (int((near_b | near_r).sum()) + 0.5) / (M * (M + 1) / 2)
+    assert n_mismatch <= int(2e-3 * cfg.Hq * M * (M + 1) // 2)
+
+
 def test_fullsize_attention_rows(full):
     cfg = full["cfg"]
     M, B, G = cfg.M, cfg.B, cfg.Hq // cfg.Hkv
@@ -133,3 +162,73 @@ def test_maximum_block_count():
     one_more = torch.empty(1, (M + 1) * B, 1, 128, dtype=torch.bfloat16, device=dev)
     with pytest.raises(RbsError, match="UNSUPPORTED"):
         rbs_block_stats(one_more, B)
+
+
+def _sampled_config_check(cfg, layers, heads_per_layer, n_rows, seed):
+    """One pass of the whole path over `cfg` on the GPU; statistics of sampled KV heads, complete mask rows and
+    attention tiles of sampled (layer, head, query block) triples are recomputed by the oracle."""
+    M, B, G = cfg.M, cfg.B, cfg.Hq // cfg.Hkv
+    Q, K, V = make_inputs(cfg)
+    dev = torch.device("cuda:0")
+    Qg, Kg, Vg = Q.to(dev), K.to(dev), V.to(dev)
+    stats = rbs_block_stats(Kg, B)
+    mask, dens, mb, mr = rbs_select(Qg, stats, B, cfg.alpha_base, cfg.alpha_rescue, cfg.n_sink, cfg.n_local,
+                                    cfg.n_recent, debug=True)
+    O, lse = rbs_sparse_prefill(Qg, Kg, Vg, mask, B, return_lse=True)
+    torch.cuda.synchronize()
+    assert rbs_device_status() == 0
+    del Qg, Kg, Vg
+    rng = np.random.default_rng(seed)
+    rq_seen = set()
+    for l in layers:
+        for h in sorted({0, cfg.Hq - 1} | {int(x) for x in rng.integers(0, cfg.Hq, size=heads_per_layer)}):
+            hk = h // G
+            K64 = to_f64(K[l, :, hk])
+            c, r = orc.block_stats(K64, B)
+            beta, lo, hi = orc.rescue_coefficient(r)
+            assert np.allclose(stats.centroid[l, hk].cpu().numpy(), c, rtol=2e-5, atol=2e-6)
+            assert np.allclose(stats.radius[l, hk].cpu().numpy(), r, rtol=2e-5)
+            assert np.allclose(stats.rq[l, hk].cpu().numpy(), [lo, hi], rtol=5e-5)
+            assert np.allclose(stats.beta[l, hk].cpu().numpy(), beta, atol=2e-4)
+            rq_seen.add((round(lo, 6), round(hi, 6)))
+            rows = sorted({0, 1, M - 1} | {int(x) for x in rng.integers(0, M, size=n_rows)})
+            Q64, V64 = to_f64(Q[l, :, h]), to_f64(V[l, :, hk])
+            sel = orc.select_head(Q64, c, r, beta, B, cfg.alpha_base, cfg.alpha_rescue, cfg.n_sink, cfg.n_local,
+                                  cfg.n_recent, rows=rows)
+            got_o, want_o, got_l, want_l = [], [], [], []
+            for i in rows:
+                near_b, near_r = sel.margin_base[i] <= 1e-3, sel.margin_rescue[i] <= 1e-3
+                assert not ((_row_bits(mb, l, h, i, M) != sel.base[i]) & ~near_b).any()
+                assert not ((_row_bits(mr, l, h, i, M) != sel.rescue[i]) & ~near_r).any()
+                got = _row_bits(mask, l, h, i, M)
+                assert not ((got != sel.final[i]) & ~(near_b | near_r)).any()
+                assert not got[i + 1:].any()
+                if i == M - 1 and M > 1024:
+                    continue                      # the dense last row of a very long sequence: covered at 128K / B 128
+                o, ls = orc.masked_attention_block(Q64, K64, V64, got, i, B)
+                want_o.append(o); want_l.append(ls)
+                t0, t1 = i * B, min(cfg.N, (i + 1) * B)
+                got_o.append(O[l, t0:t1, h].float().cpu().numpy()); got_l.append(lse[l, h, t0:t1].cpu().numpy())
+            err = np.abs(np.concatenate(got_o) - np.concatenate(want_o))
+            assert err.max() <= 2e-2 and err.mean() <= 2e-3, (l, h, err.max(), err.mean())
+            assert np.allclose(np.concatenate(got_l), np.concatenate(want_l), atol=2e-3, rtol=1e-4)
+    # density bookkeeping over the whole mask
+    words = mask.cpu().numpy().view(np.uint32)
+    pop = np.unpackbits(words.view(np.uint8)).reshape(cfg.L, cfg.Hq, -1).sum(-1)
+    assert np.array_equal(dens.cpu().numpy(), (pop / (M * (M + 1) / 2)).astype(np.float32))
+    return rq_seen
+
+
+def test_fullsize_64k_lognormal_norms():
+    """The 64K workload: needles at 5 % of the blocks and log-normal key norms (sigma 0.5), which put the radii of all
+    blocks far above the needle scale -- the case that stresses the rescue branch."""
+    _sampled_config_check(paper_configs()["q30b_64k"], layers=[0], heads_per_layer=3, n_rows=8, seed=11)
+
+
+def test_fullsize_two_layers_of_the_64_head_shape():
+    """Two consecutive layers of the 64-query / 8-KV-head shape at 128K in one call chain (batch = 2): every
+    (layer, KV head) has its own key-noise level, hence its own radius quantiles and rescue coefficients."""
+    import dataclasses
+    cfg = dataclasses.replace(paper_configs()["q32b_128k_8l"], name="q32b_128k_2l", L=2)
+    rq_seen = _sampled_config_check(cfg, layers=[0, 1], heads_per_layer=2, n_rows=5, seed=12)
+    assert len(rq_seen) >= 4            # distinct (r_low, r_high) per sampled (layer, KV head)

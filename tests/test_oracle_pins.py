@@ -198,6 +198,12 @@ def test_threshold_rule_closed_form_scene():
         assert np.array_equal(sel.base[i, :i + 1], zb >= zb.max() + math.log(a_b))
         assert np.array_equal(sel.rescue[i, :i + 1], zr >= zr.max() + math.log(a_r))
         assert not sel.base[i, i + 1:].any() and not sel.rescue[i, i + 1:].any()
+        # the margins that define the tolerance band of the GPU mask tests: the relative distance of a score from its
+        # branch threshold alpha * max S (Eq. branch_thresholds); here S_b / max S = exp(z_b - z_max) exactly, so
+        # margin = |exp(z_b - z_max) / alpha - 1|.  (Dividing by max S instead of alpha * max S would fail this.)
+        assert np.allclose(sel.margin_base[i, :i + 1], np.abs(np.exp(zb - zb.max()) / a_b - 1.0), rtol=1e-12, atol=1e-14)
+        assert np.allclose(sel.margin_rescue[i, :i + 1], np.abs(np.exp(zr - zr.max()) / a_r - 1.0), rtol=1e-12, atol=1e-14)
+        assert np.all(np.isinf(sel.margin_base[i, i + 1:])) and np.all(np.isinf(sel.margin_rescue[i, i + 1:]))
     assert not sel.forced.any()
     assert np.array_equal(sel.final, sel.base | sel.rescue)
     # the scene has rows where the rescue mask does not contain the base mask and vice versa

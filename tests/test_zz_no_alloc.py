@@ -42,6 +42,15 @@ def test_static_scratch_select_matches_workspace_select_on_two_calls_in_a_row():
         assert torch.equal(dens, want[1])
         assert torch.equal(stats.beta, beta_want) and torch.equal(stats.rq, rq_want)
         results.append(float(dens.mean()))
+        # the property the entry point exists for: a call (after the device's first one) takes no device memory --
+        # the driver reports the same free bytes before and after, with nothing handed back in between
+        free_before, _ = torch.cuda.mem_get_info(dev)
+        rbs_select_static(Qg, stats, cfg.B, cfg.alpha_base, cfg.alpha_rescue, cfg.n_sink, cfg.n_local, cfg.n_recent,
+                          mask=mask, density=dens, dbg_base=db, dbg_rescue=dr)
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info(dev)
+        assert free_after == free_before
+        assert torch.equal(mask, want[0]) and torch.equal(dens, want[1])
     assert all(0.0 < r <= 1.0 for r in results)
 
 
