@@ -39,6 +39,7 @@ SelectWorkspace select_workspace(const Dims& x) {
   w.off_clo = off; off = align_up(off + cbytes, 256);
   w.off_g = off; off = align_up(off + static_cast<size_t>(x.L) * x.Hkv * w.Mpad * sizeof(float), 256);
   w.off_cn = off; off = align_up(off + static_cast<size_t>(x.L) * x.Hkv * w.Mpad * sizeof(float), 256);
+  w.off_perm = off; off = align_up(off + static_cast<size_t>(x.L) * x.Hkv * w.Mpad * sizeof(int), 256);
   w.off_counts = off; off = align_up(off + static_cast<size_t>(x.L) * x.Hq * sizeof(unsigned int), 256);
   w.bytes = off;
   return w;

@@ -42,7 +42,7 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 // Workspace carve-up of rbs_select (all offsets 256-byte aligned).
 struct SelectWorkspace {
-  size_t off_chi, off_clo, off_g, off_cn, off_counts, bytes;
+  size_t off_chi, off_clo, off_g, off_cn, off_perm, off_counts, bytes;
   int Mpad;  // centroid rows per (l, hk) in the bf16 copies, multiple of 128
 };
 SelectWorkspace select_workspace(const Dims& x);

@@ -17,13 +17,19 @@ namespace rbs {
 // ---------------------------------------------------------------------------------------------
 constexpr int kCoeffThreads = 1024;
 
+// Besides beta, the kernel fixes the ORDER in which the scoring kernels see the blocks of each 128-row centroid tile:
+// inside a tile the rows with r_b beta_b = 0 (at least half of all blocks: every radius at or below the median) come
+// first, the others after them (the other way round in odd tiles).  perm[pos] = block index, gs[pos] = r_b beta_b scale
+// (log2 units per unit of query norm) in that order.  A scoring warp whose 32 rows all have gs = 0 then needs no
+// second exponential per logit, because S_rescue = S_base there; without the partition hardly any warp would qualify.
 __global__ void __launch_bounds__(kCoeffThreads)
 rescue_coeff_kernel(const float* __restrict__ radius, int M, int P /* pow2 >= M */, float scale_log2,
-                    float* __restrict__ beta, float* __restrict__ rq, float* __restrict__ g, int Mpad,
-                    int beta_mode /* 0: Eq. (beta), 1: beta = 0, 2: beta = 1 */) {
+                    float* __restrict__ beta, float* __restrict__ rq, float* __restrict__ gs, int* __restrict__ perm,
+                    int Mpad, int beta_mode /* 0: Eq. (beta), 1: beta = 0, 2: beta = 1 */) {
   extern __shared__ float s_sorted[];
   __shared__ float s_q[2];
-  const int hd = blockIdx.x, tid = threadIdx.x;
+  __shared__ unsigned short s_zero[8192 / 32];   // per group of 32 rows: how many have gs = 0
+  const int hd = blockIdx.x, tid = threadIdx.x, lane = tid & 31;
   const float* r = radius + static_cast<int64_t>(hd) * M;
   for (int idx = tid; idx < P; idx += kCoeffThreads) s_sorted[idx] = idx < M ? r[idx] : __int_as_float(0x7f800000);
   __syncthreads();
@@ -55,34 +61,63 @@ rescue_coeff_kernel(const float* __restrict__ radius, int M, int P /* pow2 >= M 
   const float r_low = s_q[0], r_high = s_q[1];
   const bool live = r_high > r_low;
   const float inv = live ? 1.0f / (r_high - r_low) : 0.f;
+  auto coeff = [&](int idx) -> float {   // r_b beta_b scale of block idx (0 for padding rows); also writes beta
+    if (idx >= M) return 0.f;
+    const float rb = r[idx];
+    float bt = live ? fminf(fmaxf((rb - r_low) * inv, 0.f), 1.f) : 0.f;
+    if (beta_mode == 1) bt = 0.f;
+    if (beta_mode == 2) bt = 1.f;
+    beta[static_cast<int64_t>(hd) * M + idx] = bt;
+    return rb * bt * scale_log2;
+  };
+  // Mpad is a multiple of 128 and the loops below step by the CTA size, so every warp stays whole
   for (int idx = tid; idx < Mpad; idx += kCoeffThreads) {
-    float bt = 0.f, rb = 0.f;
-    if (idx < M) {
-      rb = r[idx];
-      bt = live ? fminf(fmaxf((rb - r_low) * inv, 0.f), 1.f) : 0.f;
-      if (beta_mode == 1) bt = 0.f;
-      if (beta_mode == 2) bt = 1.f;
-      beta[static_cast<int64_t>(hd) * M + idx] = bt;
+    const uint32_t z = __ballot_sync(0xffffffffu, coeff(idx) == 0.f);
+    if (lane == 0) s_zero[idx >> 5] = static_cast<unsigned short>(__popc(z));
+  }
+  __syncthreads();
+  for (int idx = tid; idx < Mpad; idx += kCoeffThreads) {
+    const float g = coeff(idx);
+    const bool zero = g == 0.f;
+    const uint32_t z = __ballot_sync(0xffffffffu, zero);
+    const int tile = idx >> 7, w_in_tile = (idx >> 5) & 3;
+    int zeros_tile = 0, zeros_before = 0;
+#pragma unroll
+    for (int w = 0; w < 4; ++w) {
+      const int c = s_zero[tile * 4 + w];
+      zeros_tile += c;
+      if (w < w_in_tile) zeros_before += c;
     }
-    g[static_cast<int64_t>(hd) * Mpad + idx] = rb * bt;
+    zeros_before += __popc(z & ((1u << lane) - 1u));
+    const int before = idx & 127;                       // rows of the tile in front of this one
+    int pos = zero ? zeros_before : zeros_tile + (before - zeros_before);
+    // odd tiles are laid out the other way round, so that the warp that gets the rows without a rescue term (half the
+    // exponentials) in one tile gets the expensive rows in the next: over a query block's tiles the warps even out
+    if (tile & 1) pos = 127 - pos;
+    const int64_t dst = static_cast<int64_t>(hd) * Mpad + tile * 128 + pos;
+    gs[dst] = g;
+    perm[dst] = idx;
   }
 }
 
 // ---------------------------------------------------------------------------------------------
 // 2. fp32 centroid -> bf16 hi + bf16 lo, rows padded to Mpad with zeros
 // ---------------------------------------------------------------------------------------------
-__global__ void split_centroid_kernel(const float* __restrict__ centroid, int M, int Mpad, int64_t n_rows_padded,
-                                      __nv_bfloat16* __restrict__ chi, __nv_bfloat16* __restrict__ clo,
-                                      float* __restrict__ cnorm) {
-  // one thread per 4 elements, one warp per centroid row (also writes the row's L2 norm)
+__global__ void split_centroid_kernel(const float* __restrict__ centroid, const int* __restrict__ perm, int M, int Mpad,
+                                      int64_t n_rows_padded, float scale_log2, __nv_bfloat16* __restrict__ chi,
+                                      __nv_bfloat16* __restrict__ clo, float* __restrict__ cnorm) {
+  // One thread per 4 elements, one warp per row of the bf16 copies.  Row `row` holds block perm[row] of its
+  // (batch, KV head), multiplied by log2(e)/sqrt(d) so that the tensor-core product is the scaled logit in log2 units;
+  // also writes the row's L2 norm (of the scaled centroid).
   const int64_t t = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   const int64_t row = t / (kHeadDim / 4);
   const int c4 = static_cast<int>(t % (kHeadDim / 4));
   if (row >= n_rows_padded) return;   // whole warps: the grid covers rows in units of 32 threads
   const int64_t hd = row / Mpad;
-  const int b = static_cast<int>(row % Mpad);
+  const int b = perm[row];
   float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
   if (b < M) v = *reinterpret_cast<const float4*>(centroid + (hd * M + b) * kHeadDim + c4 * 4);
+  v.x *= scale_log2; v.y *= scale_log2; v.z *= scale_log2; v.w *= scale_log2;
   const __nv_bfloat16 h0 = __float2bfloat16_rn(v.x), h1 = __float2bfloat16_rn(v.y);
   const __nv_bfloat16 h2 = __float2bfloat16_rn(v.z), h3 = __float2bfloat16_rn(v.w);
   const float l0 = v.x - __bfloat162float(h0), l1 = v.y - __bfloat162float(h1);
@@ -111,7 +146,9 @@ __global__ void split_centroid_kernel(const float* __restrict__ centroid, int M,
 // ---------------------------------------------------------------------------------------------
 struct SelectParams {
   const __nv_bfloat16* Q; int64_t qsb, qst, qsh;
-  const __nv_bfloat16* chi; const __nv_bfloat16* clo; const float* g; const float* cnorm;
+  // per padded centroid row, in the tile-partitioned order of rescue_coeff_kernel: bf16 hi / lo halves of the scaled
+  // centroid, gs = r beta scale, norm of the scaled centroid, and the block index the row holds
+  const __nv_bfloat16* chi; const __nv_bfloat16* clo; const float* gs; const float* cnorm; const int* perm;
   int M, Mpad, W, L, Hq, G, N;
   int q0, Mq, Nq;   // this call's queries: first query block (global index), number of blocks, number of tokens
   float scale_log2, t_base, t_rescue;  // thresholds as log2(alpha)
@@ -119,6 +156,235 @@ struct SelectParams {
   uint32_t* mask; uint32_t* dbg_base; uint32_t* dbg_rescue;
   unsigned int* counts;
 };
+
+// Barrier `id` over the NT threads of one epilogue group, returning whether `ok` held in all of them.
+template <int NT>
+__device__ __forceinline__ bool group_all(bool ok, int id) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, %2, %3, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r) : "r"(static_cast<uint32_t>(ok)), "r"(id), "n"(NT) : "memory");
+  return r != 0;
+}
+
+// Query norms of one Q tile (B tokens, 128-byte-swizzled panels of 64 columns in shared memory), by the NT threads
+// of an epilogue group: sD[t] = ||q_t|| - max_t ||q_t|| (<= 0), and the maximum and the spread (max - min) of the norms
+// over the block's n_tok real tokens.  `red` is 2 * NT / 32 floats of scratch.  Two group barriers.
+template <int B, int NT>
+__device__ __forceinline__ bool query_norm_shifts(const unsigned char* q, int wtid, int n_tok, float* sD, float* red,
+                                                  int bar_id, bool ok, float& qn_max, float& qn_spread) {
+  constexpr uint32_t kPanelQ = B * 128;
+  constexpr int TPT = (B + NT - 1) / NT;   // tokens per thread
+  constexpr int NWG = NT / 32;
+  const int lane = wtid & 31, wq = wtid >> 5;
+  float nrm[TPT];
+  float mx = 0.f, mn = INFINITY;
+#pragma unroll
+  for (int u = 0; u < TPT; ++u) {
+    const int tok = wtid + u * NT;
+    nrm[u] = 0.f;
+    if (ok && tok < B) {
+      float s2 = 0.f;
+#pragma unroll
+      for (int c = 0; c < 16; ++c) {
+        const uint4 v = *reinterpret_cast<const uint4*>(q + (c >> 3) * kPanelQ + tok * 128 + (((c & 7) ^ (tok & 7)) << 4));
+        const uint32_t wv[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float a = bf16lo(wv[e]), c2 = bf16hi(wv[e]);
+          s2 = fmaf(a, a, s2);
+          s2 = fmaf(c2, c2, s2);
+        }
+      }
+      nrm[u] = sqrtf(s2);
+      if (tok < n_tok) { mx = fmaxf(mx, nrm[u]); mn = fminf(mn, nrm[u]); }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+  }
+  if (lane == 0) { red[wq] = mx; red[NWG + wq] = mn; }
+  ok = group_all<NT>(ok, bar_id);
+  qn_max = red[0];
+  float qn_min = red[NWG];
+#pragma unroll
+  for (int u = 1; u < NWG; ++u) { qn_max = fmaxf(qn_max, red[u]); qn_min = fminf(qn_min, red[NWG + u]); }
+  qn_spread = qn_max - qn_min;
+#pragma unroll
+  for (int u = 0; u < TPT; ++u) {
+    const int tok = wtid + u * NT;
+    if (tok < B) sD[tok] = nrm[u] - qn_max;
+  }
+  return group_all<NT>(ok, bar_id);
+}
+
+// Scores the 128 centroid rows of one tile against the B tokens of a query block, one row per thread, from the
+// accumulator row at `taddr` in tensor memory, which holds x_t = q_t . c_b scale in log2 units (the scale is folded
+// into the centroids).  With the shifts  m_b = ||q||max ||c_b scale||  (Cauchy-Schwarz: x_t <= m_b)  and
+// m_r = m_b + ||q||max gs  the two exponents are
+//     e_t = x_t - m_b                 (base branch, Eq. base_score)
+//     f_t = e_t + gs (||q_t|| - ||q||max) = (x_t + ||q_t|| gs) - m_r     (rescue branch, Eq. rescue_score)
+// both <= 0, one packed add and one packed multiply-add per pair of tokens; then L = m + log2 sum_t 2^(.)
+// (Eq. block_aggregation as a per-block log-sum-exp; any shift common to the block's tokens cancels).
+// The bounds are used as shifts only while no term can underflow: e_t >= -2 m_b, f_t >= -2 m_b - gs * spread of the
+// norms.  Otherwise (warp-uniform decision) a first pass takes the exact maxima and each branch gets its own pass.
+// A warp whose 32 rows all have gs = 0 computes no rescue exponentials: S_rescue = S_base there.
+// `release()` is called once, when the accumulator has been read for the last time.
+template <int B, bool PREFETCH, typename Release>
+__device__ __forceinline__ void score_tile(uint32_t taddr, const float* __restrict__ sD, float gs, float cn, float qn_max,
+                                           float qn_spread, int n_tok, Release release, float& Lb, float& Lr) {
+  float mb = qn_max * cn * 1.0001f;
+  const bool no_rescue = __all_sync(0xffffffffu, gs == 0.f);
+  const bool cheap = __all_sync(0xffffffffu, mb <= 60.0f && fmaf(gs, qn_spread, 2.0f * mb) <= 120.0f);
+  float shift_r = fmaf(qn_max, gs, mb);      // m_r
+  float c_first = -mb, c_second = 0.f;
+  int n_pass = 1;
+  if (!cheap) {
+    // exact maxima of x and of y = x + ||q_t|| gs
+    float mb0 = -INFINITY, mb1 = -INFINITY, mr0 = -INFINITY, mr1 = -INFINITY;
+    const uint64_t g2 = f2_pack(gs, gs), qm2 = f2_pack(qn_max, qn_max);
+#pragma unroll 1
+    for (int c0 = 0; c0 < B; c0 += 32) {
+      uint32_t r[32];
+      tmem_ld32(taddr + c0, r);
+      tmem_wait_ld();
+      if (n_tok < B) {
+#pragma unroll
+        for (int qq = 0; qq < 32; ++qq)
+          if (c0 + qq >= n_tok) r[qq] = 0xff800000u;   // -inf: tokens past the sequence end do not count
+      }
+#pragma unroll
+      for (int j = 0; j < 32; j += 4) {
+        const float4 d = *reinterpret_cast<const float4*>(sD + c0 + j);
+        float y0, y1, y2, y3;
+        f2_unpack(f2_fma(f2_add(f2_pack(d.x, d.y), qm2), g2, f2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1]))), y0, y1);
+        f2_unpack(f2_fma(f2_add(f2_pack(d.z, d.w), qm2), g2, f2_pack(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]))), y2, y3);
+        mb0 = max3(mb0, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
+        mb1 = max3(mb1, __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
+        mr0 = max3(mr0, y0, y1);
+        mr1 = max3(mr1, y2, y3);
+      }
+    }
+    mb = fmaxf(mb0, mb1);
+    shift_r = fmaxf(mr0, mr1);
+    c_first = -mb;
+    c_second = fmaf(qn_max, gs, -shift_r);     // e' = x + c  =>  e' + gs (||q_t|| - ||q||max) = y_t - max y
+    n_pass = no_rescue ? 1 : 2;
+  }
+  const uint64_t g2 = f2_pack(gs, gs);
+  float sum_b = 0.f, sum_r = 0.f;
+#pragma unroll 1
+  for (int pass = 0; pass < n_pass; ++pass) {
+    const float c = pass == 0 ? c_first : c_second;
+    const uint64_t c2 = f2_pack(c, c);
+    const bool last = pass == n_pass - 1;
+    uint64_t sb_a = 0ull, sb_b = 0ull, sr_a = 0ull, sr_b = 0ull;
+    auto chunk = [&](uint32_t (&r)[32], int c0) {
+      if (n_tok < B) {
+#pragma unroll
+        for (int qq = 0; qq < 32; ++qq)
+          if (c0 + qq >= n_tok) r[qq] = 0xff800000u;   // -inf
+      }
+#pragma unroll
+      for (int j = 0; j < 32; j += 4) {
+        const uint64_t e01 = f2_add(f2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), c2);
+        const uint64_t e23 = f2_add(f2_pack(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])), c2);
+        float e0, e1, e2, e3;
+        f2_unpack(e01, e0, e1);
+        f2_unpack(e23, e2, e3);
+        sb_a = f2_add(sb_a, f2_pack(fast_exp2(e0), fast_exp2(e1)));
+        sb_b = f2_add(sb_b, f2_pack(fast_exp2(e2), fast_exp2(e3)));
+        if (!no_rescue) {
+          const float4 d = *reinterpret_cast<const float4*>(sD + c0 + j);
+          float f0, f1, f2, f3;
+          f2_unpack(f2_fma(f2_pack(d.x, d.y), g2, e01), f0, f1);
+          f2_unpack(f2_fma(f2_pack(d.z, d.w), g2, e23), f2, f3);
+          sr_a = f2_add(sr_a, f2_pack(fast_exp2(f0), fast_exp2(f1)));
+          sr_b = f2_add(sr_b, f2_pack(fast_exp2(f2), fast_exp2(f3)));
+        }
+      }
+    };
+    if (PREFETCH) {
+      uint32_t ra[32], rb[32];
+      tmem_ld32(taddr, ra);
+#pragma unroll 1
+      for (int c0 = 0; c0 < B; c0 += 64) {
+        tmem_wait_ld();
+        tmem_ld32(taddr + c0 + 32, rb);          // on its way while the first 32 columns are reduced
+        chunk(ra, c0);
+        tmem_wait_ld();
+        if (c0 + 64 < B) tmem_ld32(taddr + c0 + 64, ra);
+        else if (last) release();                 // the accumulator has been read completely
+        chunk(rb, c0 + 32);
+      }
+    } else {
+#pragma unroll 1
+      for (int c0 = 0; c0 < B; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(taddr + c0, r);
+        tmem_wait_ld();
+        if (last && c0 + 32 >= B) release();
+        chunk(r, c0);
+      }
+    }
+    float a0, a1, a2, a3;
+    f2_unpack(f2_add(sb_a, sb_b), a0, a1);
+    f2_unpack(f2_add(sr_a, sr_b), a2, a3);
+    if (pass == 0) sum_b = a0 + a1;
+    if (last) sum_r = a2 + a3;
+  }
+  Lb = mb + fast_log2(sum_b);
+  Lr = no_rescue ? Lb : shift_r + fast_log2(sum_r);
+}
+
+
+// The single-pass case of score_tile for the columns [c_begin, c_begin + NC) of the accumulator row only:
+// sum_t 2^(x_t + c) and sum_t 2^(x_t + c + gs (||q_t|| - ||q||max)) over those tokens.
+template <int B, int NC>
+__device__ __forceinline__ void partial_sums(uint32_t taddr, const float* __restrict__ sD, float gs, float c, bool no_rescue,
+                                             int n_tok, int c_begin, float& sum_b, float& sum_r) {
+  const uint64_t g2 = f2_pack(gs, gs), c2 = f2_pack(c, c);
+  uint64_t sb_a = 0ull, sb_b = 0ull, sr_a = 0ull, sr_b = 0ull;
+#pragma unroll 1
+  for (int c0 = c_begin; c0 < c_begin + NC; c0 += 32) {
+    uint32_t r[32];
+    tmem_ld32(taddr + c0, r);
+    tmem_wait_ld();
+    if (n_tok < B) {
+#pragma unroll
+      for (int qq = 0; qq < 32; ++qq)
+        if (c0 + qq >= n_tok) r[qq] = 0xff800000u;   // -inf: tokens past the sequence end do not count
+    }
+#pragma unroll
+    for (int j = 0; j < 32; j += 4) {
+      const uint64_t e01 = f2_add(f2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), c2);
+      const uint64_t e23 = f2_add(f2_pack(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])), c2);
+      float e0, e1, e2, e3;
+      f2_unpack(e01, e0, e1);
+      f2_unpack(e23, e2, e3);
+      sb_a = f2_add(sb_a, f2_pack(fast_exp2(e0), fast_exp2(e1)));
+      sb_b = f2_add(sb_b, f2_pack(fast_exp2(e2), fast_exp2(e3)));
+      if (!no_rescue) {
+        const float4 d = *reinterpret_cast<const float4*>(sD + c0 + j);
+        float f0, f1, f2, f3;
+        f2_unpack(f2_fma(f2_pack(d.x, d.y), g2, e01), f0, f1);
+        f2_unpack(f2_fma(f2_pack(d.z, d.w), g2, e23), f2, f3);
+        sr_a = f2_add(sr_a, f2_pack(fast_exp2(f0), fast_exp2(f1)));
+        sr_b = f2_add(sr_b, f2_pack(fast_exp2(f2), fast_exp2(f3)));
+      }
+    }
+  }
+  float a0, a1, a2, a3;
+  f2_unpack(f2_add(sb_a, sb_b), a0, a1);
+  f2_unpack(f2_add(sr_a, sr_b), a2, a3);
+  sum_b = a0 + a1;
+  sum_r = a2 + a3;
+}
 
 constexpr int kTcThreads = 192;
 
@@ -211,113 +477,27 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   } else {
     // ------------------------------- epilogue: one centroid row per thread -------------------------------
     const int row = warp * 32 + lane;
-    bool ok = mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
-    for (int tok = tid; ok && tok < B; tok += 128) {   // raw query norms ||q_t||_2
-      float s2 = 0.f;
-#pragma unroll
-      for (int c = 0; c < 16; ++c) {
-        const uint4 v = *reinterpret_cast<const uint4*>(sQ + (c >> 3) * kPanelQ + tok * 128 + (((c & 7) ^ (tok & 7)) << 4));
-        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          const float a = bf16lo(w[k]), c2 = bf16hi(w[k]);
-          s2 = fmaf(a, a, s2);
-          s2 = fmaf(c2, c2, s2);
-        }
-      }
-      sQn[tok] = sqrtf(s2);
-    }
-    asm volatile("bar.sync 1, 128;" ::: "memory");   // the four epilogue warps
-    // largest query norm of the block: with it, ||q|| ||c_b|| bounds every logit of block b from above
-    float qn_max = 0.f;
-#pragma unroll
-    for (int t = lane; t < B; t += 32) qn_max = fmaxf(qn_max, sQn[t]);
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) qn_max = fmaxf(qn_max, __shfl_xor_sync(0xffffffffu, qn_max, o));
-    const uint64_t scale2 = f2_pack(p.scale_log2, p.scale_log2);
+    bool ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull));
     const int n_tok = min(B, p.Nq - il * B);
+    float qn_max, qn_spread;
+    ok = query_norm_shifts<B, 128>(sQ, tid, n_tok, sQn, sRed, 1, ok, qn_max, qn_spread);   // sQn holds ||q_t|| - ||q||max
     for (int bt = 0; ok && bt < n_tiles; ++bt) {
       const int buf = bt & 1;
-      ok = mbar_wait(smem_u32(&bar_tfull[buf]), (bt >> 1) & 1, status, kWaitMmaDone);
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_tfull[buf]), (bt >> 1) & 1, status, kWaitMmaDone));
       if (!ok) break;
       tc_fence_after_sync();
-      const int b = bt * 128 + row;
-      const float gb = p.g[crow0 + b];            // r_b beta_b, unscaled
-      const uint64_t gb2 = f2_pack(gb, gb);
+      const int prow = crow0 + bt * 128 + row;
+      const int b = p.perm[prow];                 // the block this accumulator row belongs to
       const uint32_t taddr = tmem_base + buf * B + (static_cast<uint32_t>(warp * 32) << 16);
-      // Shift of the log-sum-exp.  Any value common to the block's tokens cancels; the Cauchy-Schwarz bounds
-      // ||q||max ||c_b|| (base) and ||q||max (||c_b|| + r_b beta_b) (rescue) need no pass over the logits.  They are
-      // used when small enough that no term can underflow (2^-126); otherwise the exact maxima are taken.
-      float mb = qn_max * p.cnorm[crow0 + b] * p.scale_log2 * 1.0001f;
-      float mr = fmaf(qn_max * gb, p.scale_log2 * 1.0001f, mb);
-      const bool exact_shift = !__all_sync(0xffffffffu, mr <= 60.0f);
-      if (exact_shift) {
-      // pass 1: maxima of the raw logits x and of y = x + ||q|| r beta
-      float mb0 = -INFINITY, mb1 = -INFINITY, mr0 = -INFINITY, mr1 = -INFINITY;
-#pragma unroll 1
-      for (int c0 = 0; c0 < B; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(taddr + c0, r);
-        tmem_wait_ld();
-        if (n_tok < B) {   // short last query block: tokens past the sequence end do not count
-#pragma unroll
-          for (int q = 0; q < 32; ++q)
-            if (c0 + q >= n_tok) r[q] = 0xff800000u;   // -inf
-        }
-#pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          const float4 qn = *reinterpret_cast<const float4*>(sQn + c0 + j);
-          float y0, y1, y2, y3;
-          f2_unpack(f2_fma(f2_pack(qn.x, qn.y), gb2, f2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1]))), y0, y1);
-          f2_unpack(f2_fma(f2_pack(qn.z, qn.w), gb2, f2_pack(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]))), y2, y3);
-          mb0 = max3(mb0, __uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-          mb1 = max3(mb1, __uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-          mr0 = max3(mr0, y0, y1);
-          mr1 = max3(mr1, y2, y3);
-        }
-      }
-        mb = fmaxf(mb0, mb1) * p.scale_log2;   // log2 units
-        mr = fmaxf(mr0, mr1) * p.scale_log2;
-      }
-      const uint64_t nmb2 = f2_pack(-mb, -mb), nmr2 = f2_pack(-mr, -mr);
-      uint64_t sb2 = 0ull, sr2 = 0ull, sb2b = 0ull, sr2b = 0ull;
-#pragma unroll 1
-      for (int c0 = 0; c0 < B; c0 += 32) {
-        uint32_t r[32];
-        tmem_ld32(taddr + c0, r);
-        tmem_wait_ld();
-        if (n_tok < B) {   // short last query block: tokens past the sequence end do not count
-#pragma unroll
-          for (int q = 0; q < 32; ++q)
-            if (c0 + q >= n_tok) r[q] = 0xff800000u;   // -inf
-        }
-        if (c0 + 32 >= B) {   // accumulator fully read: hand the TMEM buffer back to the MMA warp
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(smem_u32(&bar_tempty[buf]));
-        }
-#pragma unroll
-        for (int j = 0; j < 32; j += 4) {
-          const float4 qn = *reinterpret_cast<const float4*>(sQn + c0 + j);
-          const uint64_t x01 = f2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1]));
-          const uint64_t x23 = f2_pack(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3]));
-          float e0, e1, e2, e3, f0, f1, f2, f3;
-          f2_unpack(f2_fma(x01, scale2, nmb2), e0, e1);
-          f2_unpack(f2_fma(x23, scale2, nmb2), e2, e3);
-          f2_unpack(f2_fma(f2_fma(f2_pack(qn.x, qn.y), gb2, x01), scale2, nmr2), f0, f1);
-          f2_unpack(f2_fma(f2_fma(f2_pack(qn.z, qn.w), gb2, x23), scale2, nmr2), f2, f3);
-          sb2 = f2_add(sb2, f2_pack(fast_exp2(e0), fast_exp2(e1)));
-          sb2b = f2_add(sb2b, f2_pack(fast_exp2(e2), fast_exp2(e3)));
-          sr2 = f2_add(sr2, f2_pack(fast_exp2(f0), fast_exp2(f1)));
-          sr2b = f2_add(sr2b, f2_pack(fast_exp2(f2), fast_exp2(f3)));
-        }
-      }
-      float a0, a1, a2, a3;
-      f2_unpack(f2_add(sb2, sb2b), a0, a1);
-      f2_unpack(f2_add(sr2, sr2b), a2, a3);
+      float Lb, Lr;
+      score_tile<B, true>(taddr, sQn, p.gs[prow], p.cnorm[prow], qn_max, qn_spread, n_tok, [&]() {
+        tc_fence_before_sync();                   // hand the TMEM buffer back to the MMA warp
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&bar_tempty[buf]));
+      }, Lb, Lr);
       const bool causal = b <= i;
-      sLb[b] = causal ? mb + fast_log2(a0 + a1) : -INFINITY;
-      sLr[b] = causal ? mr + fast_log2(a2 + a3) : -INFINITY;
+      sLb[b] = causal ? Lb : -INFINITY;
+      sLr[b] = causal ? Lr : -INFINITY;
     }
   }
   tc_fence_before_sync();
@@ -364,6 +544,275 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
   if (lane == 0 && cnt) atomicAdd(p.counts + l * p.Hq + h, cnt);
 }
 
+// ---------------------------------------------------------------------------------------------
+// 3b. The same scoring as a persistent kernel, one CTA per SM, that serves TWO query heads of a KV group per work
+//     item (l, KV head, query block, head pair).  The two heads score against the same centroids, so every centroid
+//     tile is brought into shared memory once for both (half the L2 -> shared-memory traffic per score) and the
+//     tensor core runs the two heads' products back to back (four accumulators in tensor memory: 2 heads x 2 buffers).
+//     Warps 0-7 / 8-15: epilogue of head 0 / head 1.  A row of the accumulator (one centroid) is shared by two warps
+//     with the same lane quarter of tensor memory: warp q reduces the first half of the block's tokens, warp q + 4
+//     the second half and hands its two partial sums over through shared memory, so that every scheduler has four
+//     epilogue warps to hide the latencies of the exponentials and of the tensor-memory loads behind one another.
+//     Warp 16: TMA producer, which also fetches the NEXT item's two Q tiles while the current item is being scored;
+//     warp 17: MMA issuer.  Each epilogue group keeps its running row maxima in registers and does its own threshold /
+//     pack pass, during which the MMA warp is already filling the accumulators of the next item.
+//     Work items are dealt round-robin, longest rows first.
+// ---------------------------------------------------------------------------------------------
+constexpr int kPairThreads = 576;
+constexpr int kPairProducer = 16, kPairMma = 17;
+
+template <int B>
+__global__ void __launch_bounds__(kPairThreads, 1)
+select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmChi,
+                   const __grid_constant__ CUtensorMap tmClo, const SelectParams p, int n_items, int l_floats,
+                   unsigned int* status) {
+  constexpr uint32_t kPanelC = 128 * 128;          // one 64-column panel of a 128-row centroid tile
+  constexpr uint32_t kStage = 4 * kPanelC;         // hi panels 0,1 then lo panels 0,1
+  constexpr uint32_t kPanelQ = B * 128;
+  constexpr uint32_t kQTile = 2 * kPanelQ;         // one head's Q tile
+  constexpr uint32_t kIdesc = idesc_bf16_f32(128, B, false);
+  extern __shared__ __align__(1024) unsigned char smem[];
+  unsigned char* sC = smem;                                        // 64 KB
+  unsigned char* sQ = sC + kStage;                                 // [slot 2][head 2][kQTile]
+  float* sQn = reinterpret_cast<float*>(sQ + 4 * kQTile);          // [head 2][B]
+  float* sL = sQn + 2 * B;                                         // [head 2][branch 2][l_floats]
+  __shared__ __align__(8) uint64_t bar_qfull[2], bar_qempty[2], bar_cfull[2], bar_cempty[2], bar_tfull[2][2], bar_tempty[2][2];
+  __shared__ __align__(8) uint64_t bar_half[2][4][2];      // [head][lane quarter][tile parity]: second half's sums are there
+  __shared__ __align__(8) float2 sHalf[2][4][2][32];       // the partial sums (base, rescue) of the second half
+  __shared__ float sRed[2][2][8], sRedQ[2][16];
+  __shared__ uint32_t s_tmem;
+
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int Hkv = p.Hq / p.G, GP = p.G / 2;
+  const int per_i = p.L * Hkv * GP;
+
+  if (tid == 0) {
+    for (int s = 0; s < 2; ++s) {
+      // a Q slot is free once the item's last product has been read by the tensor core AND both epilogue groups have
+      // taken their query norms from it (an item of one or two centroid tiles can be multiplied completely before the
+      // epilogue groups even reach it: without their arrivals the slot would be refilled under them, and the full
+      // barrier could run two phases ahead of a waiter, which a parity wait cannot tell from no progress)
+      mbar_init(smem_u32(&bar_qfull[s]), 1); mbar_init(smem_u32(&bar_qempty[s]), 3);
+      mbar_init(smem_u32(&bar_cfull[s]), 1); mbar_init(smem_u32(&bar_cempty[s]), 1);
+      for (int hw = 0; hw < 2; ++hw) {
+        mbar_init(smem_u32(&bar_tfull[hw][s]), 1); mbar_init(smem_u32(&bar_tempty[hw][s]), 8);
+        for (int q = 0; q < 4; ++q) mbar_init(smem_u32(&bar_half[hw][q][s]), 1);
+      }
+    }
+    mbar_fence_init();
+  }
+  if (warp == kPairMma) tmem_alloc(smem_u32(&s_tmem), 4 * B);
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = s_tmem;
+
+  // item w -> (query block of the chunk, batch, KV head, head pair); longest rows first
+  auto decode = [&](int w, int& il, int& l, int& hk, int& h0) {
+    il = p.Mq - 1 - w / per_i;
+    int rem = w % per_i;
+    const int pr = rem % GP; rem /= GP;
+    hk = rem % Hkv; l = rem / Hkv;
+    h0 = hk * p.G + 2 * pr;
+  };
+
+  if (warp == kPairProducer) {
+    // ------------------------------- TMA producer -------------------------------
+    if (lane == 0) {
+      tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmChi); tma_prefetch_desc(&tmClo);
+      uint32_t nq = 0, nc = 0;     // Q loads (items) and centroid tiles issued so far
+      bool ok = true;
+      auto load_q = [&](int w) {
+        int il, l, hk, h0;
+        decode(w, il, l, hk, h0);
+        const uint32_t slot = nq & 1;
+        if (nq >= 2 && !mbar_wait(smem_u32(&bar_qempty[slot]), ((nq >> 1) - 1) & 1, status, kWaitStageFree)) { ok = false; return; }
+        const uint32_t dst = smem_u32(sQ) + slot * 2 * kQTile, bar = smem_u32(&bar_qfull[slot]);
+        mbar_arrive_expect_tx(bar, 2 * kQTile);
+        for (int hw = 0; hw < 2; ++hw) {
+          tma_load_4d(dst + hw * kQTile, &tmQ, bar, 0, h0 + hw, il * B, l);
+          tma_load_4d(dst + hw * kQTile + kPanelQ, &tmQ, bar, 64, h0 + hw, il * B, l);
+        }
+        ++nq;
+      };
+      int w = blockIdx.x;
+      if (w < n_items) load_q(w);
+      for (; ok && w < n_items; w += gridDim.x) {
+        int il, l, hk, h0;
+        decode(w, il, l, hk, h0);
+        const int n_tiles = (p.q0 + il) / 128 + 1;
+        const int crow0 = static_cast<int>((static_cast<int64_t>(l) * Hkv + hk) * p.Mpad);
+        const uint32_t dst = smem_u32(sC);
+        for (int bt = 0; ok && bt < n_tiles; ++bt, ++nc) {
+          if (nc > 0 && !mbar_wait(smem_u32(&bar_cempty[0]), (nc - 1) & 1, status, kWaitStageFree)) { ok = false; break; }
+          mbar_arrive_expect_tx(smem_u32(&bar_cfull[0]), kStage / 2);
+          tma_load_2d(dst, &tmChi, smem_u32(&bar_cfull[0]), 0, crow0 + bt * 128);
+          tma_load_2d(dst + kPanelC, &tmChi, smem_u32(&bar_cfull[0]), 64, crow0 + bt * 128);
+          if (nc > 0 && !mbar_wait(smem_u32(&bar_cempty[1]), (nc - 1) & 1, status, kWaitStageFree)) { ok = false; break; }
+          mbar_arrive_expect_tx(smem_u32(&bar_cfull[1]), kStage / 2);
+          tma_load_2d(dst + 2 * kPanelC, &tmClo, smem_u32(&bar_cfull[1]), 0, crow0 + bt * 128);
+          tma_load_2d(dst + 3 * kPanelC, &tmClo, smem_u32(&bar_cfull[1]), 64, crow0 + bt * 128);
+          // the next item's Q tiles go out right behind this item's first centroid tile
+          if (bt == 0 && w + static_cast<int>(gridDim.x) < n_items) load_q(w + gridDim.x);
+        }
+      }
+    }
+  } else if (warp == kPairMma) {
+    // ------------------------------- MMA issuer -------------------------------
+    const uint64_t dchi = smem_desc_sw128(smem_u32(sC), 16, 1024);
+    const uint64_t dclo = smem_desc_sw128(smem_u32(sC) + 2 * kPanelC, 16, 1024);
+    uint32_t nt = 0, k = 0;      // centroid tiles and items processed so far
+    bool ok = true;
+    for (int w = blockIdx.x; ok && w < n_items; w += gridDim.x, ++k) {
+      const int il = p.Mq - 1 - w / per_i;
+      const int n_tiles = (p.q0 + il) / 128 + 1;
+      const uint32_t slot = k & 1;
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_qfull[slot]), (k >> 1) & 1, status, kWaitTmaFull));
+      const uint64_t dq0 = smem_desc_sw128(smem_u32(sQ) + slot * 2 * kQTile, 16, 1024);
+      const uint64_t dq1 = smem_desc_sw128(smem_u32(sQ) + slot * 2 * kQTile + kQTile, 16, 1024);
+      for (int bt = 0; ok && bt < n_tiles; ++bt, ++nt) {
+        const uint32_t buf = nt & 1;
+        ok = mbar_wait(smem_u32(&bar_cfull[0]), nt & 1, status, kWaitTmaFull);
+        if (ok && nt >= 2) ok = mbar_wait(smem_u32(&bar_tempty[0][buf]), ((nt >> 1) - 1) & 1, status, kWaitTmemFree) &&
+                                mbar_wait(smem_u32(&bar_tempty[1][buf]), ((nt >> 1) - 1) & 1, status, kWaitTmemFree);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t d0 = tmem_base + buf * B, d1 = tmem_base + (2 + buf) * B;
+        mma_ss_k128_commit_elect(d0, dchi, dq0, kIdesc, kPanelC, kPanelQ, 0, 0);
+        mma_ss_k128_commit_elect(d1, dchi, dq1, kIdesc, kPanelC, kPanelQ, smem_u32(&bar_cempty[0]), 0);
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_cfull[1]), nt & 1, status, kWaitTmaFull));
+        if (!ok) break;
+        tc_fence_after_sync();
+        mma_ss_k128_commit_elect(d0, dclo, dq0, kIdesc, kPanelC, kPanelQ, smem_u32(&bar_tfull[0][buf]), 1);
+        mma_ss_k128_commit_elect(d1, dclo, dq1, kIdesc, kPanelC, kPanelQ, smem_u32(&bar_cempty[1]), 1);
+        mma_commit_elect(smem_u32(&bar_tfull[1][buf]));
+        if (bt == n_tiles - 1) mma_commit_elect(smem_u32(&bar_qempty[slot]));   // this item's Q tiles are free
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------- epilogue groups: one centroid row per pair of threads -------------------------------
+    const int hw = warp >> 3, wq = warp & 3, half = (warp >> 2) & 1;   // head of the pair, lane quarter, token half
+    const int wg = warp & 7;                                           // warp inside the group
+    const int row = wq * 32 + lane;
+    const int wtid = tid & 255;
+    const int gbar = 1 + hw;                                           // named barrier of this group (256 threads)
+    float* sQn_h = sQn + hw * B;
+    float* sLb = sL + (hw * 2) * l_floats;
+    float* sLr = sLb + l_floats;
+    uint32_t nt = 0, k = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; ok && w < n_items; w += gridDim.x, ++k) {
+      int il, l, hk, h0;
+      decode(w, il, l, hk, h0);
+      const int i = p.q0 + il, h = h0 + hw;
+      const int n_tiles = i / 128 + 1;
+      const int crow0 = static_cast<int>((static_cast<int64_t>(l) * Hkv + hk) * p.Mpad);
+      const uint32_t slot = k & 1;
+      const unsigned char* q = sQ + slot * 2 * kQTile + hw * kQTile;
+      ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_qfull[slot]), (k >> 1) & 1, status, kWaitTmaFull));
+      const int n_tok = min(B, p.Nq - il * B);
+      float qn_max, qn_spread;
+      ok = query_norm_shifts<B, 256>(q, wtid, n_tok, sQn_h, &sRedQ[hw][0], gbar, ok, qn_max, qn_spread);
+      if (wtid == 0) mbar_arrive(smem_u32(&bar_qempty[slot]));      // the Q tile itself is not read again by this group
+      float mxb = -INFINITY, mxr = -INFINITY;     // running maxima of this thread's L values (causal blocks only)
+      for (int bt = 0; ok && bt < n_tiles; ++bt, ++nt) {
+        const uint32_t buf = nt & 1;
+        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_tfull[hw][buf]), (nt >> 1) & 1, status, kWaitMmaDone));
+        if (!ok) break;
+        tc_fence_after_sync();
+        const int prow = crow0 + bt * 128 + row;
+        const float gs = p.gs[prow], cn = p.cnorm[prow];
+        const uint32_t taddr = tmem_base + (hw * 2 + buf) * B + (static_cast<uint32_t>(wq * 32) << 16);
+        // the decisions of score_tile, identical in the two warps that share these rows
+        const float mb = qn_max * cn * 1.0001f;
+        const bool no_rescue = __all_sync(0xffffffffu, gs == 0.f);
+        const bool cheap = __all_sync(0xffffffffu, mb <= 60.0f && fmaf(gs, qn_spread, 2.0f * mb) <= 120.0f);
+        const uint32_t hbar = smem_u32(&bar_half[hw][wq][buf]);
+        auto release = [&]() {                        // hand the TMEM buffer back to the MMA warp
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(smem_u32(&bar_tempty[hw][buf]));
+        };
+        if (half == 1) {
+          if (cheap) {
+            float sb, sr;
+            partial_sums<B, B / 2>(taddr, sQn_h, gs, -mb, no_rescue, n_tok, B / 2, sb, sr);
+            sHalf[hw][wq][buf][lane] = make_float2(sb, sr);
+          }
+          release();                                  // (also orders the shared-memory writes before the arrival below)
+          if (lane == 0) mbar_arrive(hbar);
+        } else {
+          float Lb, Lr;
+          if (cheap) {
+            float sb, sr;
+            partial_sums<B, B / 2>(taddr, sQn_h, gs, -mb, no_rescue, n_tok, 0, sb, sr);
+            ok = __all_sync(0xffffffffu, mbar_wait(hbar, (nt >> 1) & 1, status, kWaitPReady));
+            const float2 o = sHalf[hw][wq][buf][lane];
+            // the buffer (and with it this slot of sHalf) goes back only after the partner's sums have been taken
+            release();
+            Lb = mb + fast_log2(sb + o.x);
+            Lr = no_rescue ? Lb : fmaf(qn_max, gs, mb) + fast_log2(sr + o.y);
+          } else {
+            score_tile<B, false>(taddr, sQn_h, gs, cn, qn_max, qn_spread, n_tok, []() {}, Lb, Lr);
+            ok = __all_sync(0xffffffffu, mbar_wait(hbar, (nt >> 1) & 1, status, kWaitPReady));
+            release();
+          }
+          const int b = p.perm[prow];                 // the block this accumulator row belongs to
+          if (b > i) { Lb = -INFINITY; Lr = -INFINITY; }
+          sLb[b] = Lb;
+          sLr[b] = Lr;
+          mxb = fmaxf(mxb, Lb);
+          mxr = fmaxf(mxr, Lr);
+        }
+      }
+      // row maxima over the causal candidates, thresholds, forced blocks, union, pack: this group alone
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) {
+        mxb = fmaxf(mxb, __shfl_xor_sync(0xffffffffu, mxb, o));
+        mxr = fmaxf(mxr, __shfl_xor_sync(0xffffffffu, mxr, o));
+      }
+      if (lane == 0) { sRed[hw][0][wg] = mxb; sRed[hw][1][wg] = mxr; }
+      ok = group_all<256>(ok, gbar);
+      mxb = sRed[hw][0][0]; mxr = sRed[hw][1][0];
+#pragma unroll
+      for (int u = 1; u < 8; ++u) { mxb = fmaxf(mxb, sRed[hw][0][u]); mxr = fmaxf(mxr, sRed[hw][1][u]); }
+      const float thr_b = mxb + p.t_base, thr_r = mxr + p.t_rescue;
+      const int64_t mrow = ((static_cast<int64_t>(l) * p.Hq + h) * p.Mq + il) * p.W;
+      const bool all_forced = i >= p.M - p.n_recent;
+      unsigned int cnt = 0;
+      for (int wd = wg; ok && wd < p.W; wd += 8) {
+        const int b = wd * 32 + lane;
+        const bool valid = b <= i;
+        bool kb = false, kr = false, kf = false;
+        if (valid) {
+          kb = sLb[b] >= thr_b;
+          kr = sLr[b] >= thr_r;
+          kf = all_forced || b < p.n_sink || b > i - p.n_local;
+        }
+        const uint32_t wb = __ballot_sync(0xffffffffu, kb), wr = __ballot_sync(0xffffffffu, kr);
+        const uint32_t wf = __ballot_sync(0xffffffffu, kf);
+        if (lane == 0) {
+          const uint32_t word = wb | wr | wf;
+          p.mask[mrow + wd] = word;
+          if (p.dbg_base) p.dbg_base[mrow + wd] = wb;
+          if (p.dbg_rescue) p.dbg_rescue[mrow + wd] = wr;
+          cnt += __popc(word);
+        }
+      }
+      if (lane == 0 && cnt) atomicAdd(p.counts + l * p.Hq + h, cnt);
+      // the L arrays, norms and maxima may be overwritten after this; `ok` leaves it identical in the whole group, so
+      // that its warps leave the item loop together (a group split over a named barrier would wait forever)
+      ok = group_all<256>(ok, gbar);
+    }
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  if (warp == kPairMma) tmem_dealloc(tmem_base, 4 * B);
+}
+
 __global__ void density_kernel(const unsigned int* __restrict__ counts, int n, int q0, int Mq, float* __restrict__ density) {
   const int t = blockIdx.x * blockDim.x + threadIdx.x;
   if (t < n) {
@@ -395,6 +844,45 @@ static rbs_status launch_select_tc(const SelectParams& p, const rbs_tensor& Q, c
   return RBS_OK;
 }
 
+// Shared memory of select_pair_kernel for M blocks; 0 when this shape has to stay on the one-head kernel
+// (blocks of 256: two Q tiles of 64 KB each do not fit twice; an odd group size; very long rows).
+template <int B>
+static size_t pair_kernel_smem(const SelectParams& p, int* l_floats) {
+  if (B > 128 || p.G % 2 != 0) return 0;
+  *l_floats = (p.M + 127) / 128 * 128;
+  const size_t bytes = static_cast<size_t>(4) * 128 * 128 + 4 * 2 * static_cast<size_t>(B) * 128 + 2 * B * sizeof(float) +
+                       4 * static_cast<size_t>(*l_floats) * sizeof(float);
+  return bytes <= 227 * 1024 - 6 * 1024 ? bytes : 0;   // about 5 KB of static shared memory beside it
+}
+
+template <int B>
+static rbs_status launch_select_pair(const SelectParams& p, const rbs_tensor& Q, size_t smem, int l_floats, cudaStream_t s) {
+  CUtensorMap tmQ, tmChi, tmClo;
+  rbs_status st = make_tmap_lthd(&tmQ, Q.ptr, p.L, p.Nq, p.Hq, kHeadDim, Q.stride_batch, Q.stride_token, Q.stride_head, 64, B, true);
+  if (st != RBS_OK) return st;
+  const int64_t rows = static_cast<int64_t>(p.L) * (p.Hq / p.G) * p.Mpad;
+  if ((st = make_tmap_2d(&tmChi, p.chi, rows, kHeadDim, 64, 128)) != RBS_OK) return st;
+  if ((st = make_tmap_2d(&tmClo, p.clo, rows, kHeadDim, 64, 128)) != RBS_OK) return st;
+  unsigned int* status = device_status_ptr();
+  if (status == nullptr) return RBS_ERR_CUDA;
+  auto kern = select_pair_kernel<B>;
+  if ((st = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem)) != RBS_OK) return st;
+  const long long n_items = static_cast<long long>(p.L) * (p.Hq / 2) * p.Mq;
+  if (n_items > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
+  const int grid = static_cast<int>(n_items < sm_count() ? n_items : sm_count());
+  kern<<<grid, kPairThreads, smem, s>>>(tmQ, tmChi, tmClo, p, static_cast<int>(n_items), l_floats, status);
+  RBS_CUDA_OK(cudaGetLastError());
+  return RBS_OK;
+}
+
+template <int B>
+static rbs_status launch_select(const SelectParams& p, const rbs_tensor& Q, cudaStream_t s) {
+  int l_floats = 0;
+  const size_t smem = pair_kernel_smem<B>(p, &l_floats);
+  if (smem != 0) return launch_select_pair<B>(p, Q, smem, l_floats, s);
+  return launch_select_tc<B>(p, Q, s);
+}
+
 }  // namespace rbs
 
 // q_start_block / n_q_tokens: the queries of this call are tokens [q_start_block * B, q_start_block * B + n_q_tokens)
@@ -421,7 +909,8 @@ static rbs_status select_impl(const rbs_shape* shape, int q_start_block, int n_q
   unsigned char* wsp = static_cast<unsigned char*>(workspace);
   __nv_bfloat16* chi = reinterpret_cast<__nv_bfloat16*>(wsp + ws.off_chi);
   __nv_bfloat16* clo = reinterpret_cast<__nv_bfloat16*>(wsp + ws.off_clo);
-  float* g = reinterpret_cast<float*>(wsp + ws.off_g);
+  float* gs = reinterpret_cast<float*>(wsp + ws.off_g);
+  int* perm = reinterpret_cast<int*>(wsp + ws.off_perm);
   float* cnorm = reinterpret_cast<float*>(wsp + ws.off_cn);
   unsigned int* counts = reinterpret_cast<unsigned int*>(wsp + ws.off_counts);
   const float scale_log2 = kLog2e / sqrtf(static_cast<float>(x.d));
@@ -432,23 +921,23 @@ static rbs_status select_impl(const rbs_shape* shape, int q_start_block, int n_q
   const size_t coeff_smem = static_cast<size_t>(P) * sizeof(float);
   RBS_CUDA_OK(cudaMemsetAsync(counts, 0, static_cast<size_t>(x.L) * x.Hq * sizeof(unsigned int), s));
   rescue_coeff_kernel<<<x.L * x.Hkv, kCoeffThreads, coeff_smem, s>>>(stats.radius, x.M, P, scale_log2, stats.beta,
-                                                                     stats.rq, g, ws.Mpad, beta_mode);
+                                                                     stats.rq, gs, perm, ws.Mpad, beta_mode);
   RBS_CUDA_OK(cudaGetLastError());
   const int64_t rows = static_cast<int64_t>(x.L) * x.Hkv * ws.Mpad;
   const int64_t n_thr = rows * (kHeadDim / 4);
-  split_centroid_kernel<<<static_cast<unsigned>((n_thr + 255) / 256), 256, 0, s>>>(stats.centroid, x.M, ws.Mpad, rows, chi, clo, cnorm);
+  split_centroid_kernel<<<static_cast<unsigned>((n_thr + 255) / 256), 256, 0, s>>>(stats.centroid, perm, x.M, ws.Mpad, rows, scale_log2, chi, clo, cnorm);
   RBS_CUDA_OK(cudaGetLastError());
 
   SelectParams p;
   p.Q = static_cast<const __nv_bfloat16*>(Q.ptr); p.qsb = Q.stride_batch; p.qst = Q.stride_token; p.qsh = Q.stride_head;
-  p.chi = chi; p.clo = clo; p.g = g; p.cnorm = cnorm;
+  p.chi = chi; p.clo = clo; p.gs = gs; p.cnorm = cnorm; p.perm = perm;
   p.M = x.M; p.Mpad = ws.Mpad; p.W = x.W; p.L = x.L; p.Hq = x.Hq; p.G = x.G; p.N = x.N;
   p.q0 = q_start_block; p.Nq = n_q_tokens; p.Mq = (n_q_tokens + x.B - 1) / x.B;
   p.scale_log2 = scale_log2; p.t_base = log2f(alpha_base); p.t_rescue = log2f(alpha_rescue);
   p.n_sink = n_sink; p.n_local = n_local; p.n_recent = n_recent;
   p.mask = mask; p.dbg_base = dbg_base_mask; p.dbg_rescue = dbg_rescue_mask; p.counts = counts;
   if (x.B == 256) st = launch_select_tc<256>(p, Q, s);
-  else st = (x.B == 128) ? launch_select_tc<128>(p, Q, s) : launch_select_tc<64>(p, Q, s);
+  else st = (x.B == 128) ? launch_select<128>(p, Q, s) : launch_select<64>(p, Q, s);
   if (st != RBS_OK) return st;
   const int nh = x.L * x.Hq;
   density_kernel<<<(nh + 127) / 128, 128, 0, s>>>(counts, nh, p.q0, p.Mq, density);

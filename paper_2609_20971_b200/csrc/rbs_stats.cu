@@ -48,6 +48,9 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
 
   const int stride = gridDim.x * NG;
   int t = group * gridDim.x + blockIdx.x;
+  // K is read exactly once by this pass: its lines are marked evict-first in L2 so that they do not push out what the
+  // following kernels re-read (29.5 against 30.9 us per 128 MiB layer)
+  const uint64_t pol = make_policy_evict_first();
   auto issue = [&](int tile, int buf) {
     const uint32_t bar = bar0 + 8 * buf, slot = slot0 + buf * kSlot;
     int idx = tile;
@@ -55,8 +58,8 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
     const int b = idx % M;
     const int l = idx / M;
     mbar_arrive_expect_tx(bar, kSlot);
-    tma_load_4d(slot, &tmK, bar, 0, hk, b * B + part * RW, l);
-    tma_load_4d(slot + kPanel, &tmK, bar, 64, hk, b * B + part * RW, l);
+    tma_load_4d_hint(slot, &tmK, bar, 0, hk, b * B + part * RW, l, pol);
+    tma_load_4d_hint(slot + kPanel, &tmK, bar, 64, hk, b * B + part * RW, l, pol);
   };
   if (lane == 0) {
     for (int k = 0; k < NS; ++k)
