@@ -36,7 +36,7 @@ NCU_TRAFFIC_BYTES = {
 NOMINAL_BF16_TFLOPS = 2250.0     # dense bf16 per B200, for context next to the measured peak
 TARGET_TENSOR_FRAC = 0.60        # select + sparse attention on the selected FLOPs, of the measured bf16 peak
 TARGET_HBM_FRAC = 0.70           # statistics pass, of the measured copy bandwidth
-# kernels per step of the path: block_stats; rescue_coeff, split_centroid, select_tc, density; prefill
+# kernels per step of the path: block_stats; rescue_coeff, split_centroid, select_pair, density; prefill_tc
 LAUNCHES_PER_STEP = 6
 # the bounded oracle sample both arms time (the same in `cpu_baseline` and in `--impl reference`)
 ORACLE_SAMPLE = dict(n_heads=4, n_att_rows=48)
@@ -231,7 +231,7 @@ def replica_seed(base_seed: int, rank: int) -> int:
 # ------------------------------------------------------------------------------------------------
 # the other workloads of the benchmark plan (reported under `detail`, outside the headline's timed region)
 # ------------------------------------------------------------------------------------------------
-def time_select_sparse(Qg, Kg, Vg, Og, stats, mask, density, ws, B, sel_args, reps=3):
+def time_select_sparse(Qg, Kg, Vg, Og, stats, mask, density, ws, B, sel_args, reps=3, ws_att=None):
     """Mean ms of rbs_select and of rbs_sparse_prefill over `reps` repetitions after one warm-up."""
     from paper_2609_20971_b200 import rbs_select, rbs_sparse_prefill
     stream = torch.cuda.current_stream()
@@ -241,7 +241,7 @@ def time_select_sparse(Qg, Kg, Vg, Og, stats, mask, density, ws, B, sel_args, re
         ev[0].record(stream)
         rbs_select(Qg, stats, B, *sel_args, mask=mask, density=density, workspace=ws)
         ev[1].record(stream)
-        rbs_sparse_prefill(Qg, Kg, Vg, mask, B, out=Og)
+        rbs_sparse_prefill(Qg, Kg, Vg, mask, B, out=Og, workspace=ws_att)
         ev[2].record(stream)
         if rep > 0:
             evs.append(ev)
@@ -305,7 +305,10 @@ def measure_extra_workload(cfg, dev, peaks, with_dense=True):
     stats = alloc_stats(Kg, B)
     mask = torch.empty(L, cfg.Hq, M, (M + 31) // 32, dtype=torch.int32, device=dev)
     density = torch.empty(L, cfg.Hq, dtype=torch.float32, device=dev)
-    ws = torch.empty(workspace_bytes(RBS_OP_SELECT, RbsShape(L, cfg.N, cfg.Hq, cfg.Hkv, cfg.d, B)), dtype=torch.uint8, device=dev)
+    from paper_2609_20971_b200.binding import RBS_OP_SPARSE_PREFILL
+    shape = RbsShape(L, cfg.N, cfg.Hq, cfg.Hkv, cfg.d, B)
+    ws = torch.empty(workspace_bytes(RBS_OP_SELECT, shape), dtype=torch.uint8, device=dev)
+    ws_att = torch.empty(max(256, workspace_bytes(RBS_OP_SPARSE_PREFILL, shape)), dtype=torch.uint8, device=dev)
     sel_args = (cfg.alpha_base, cfg.alpha_rescue, cfg.n_sink, cfg.n_local, cfg.n_recent)
     t_stats, _ = time_stats_rotating(Kg, B, stats)
     rbs_block_stats(Kg, B, stats)
@@ -341,7 +344,7 @@ def measure_extra_workload(cfg, dev, peaks, with_dense=True):
 def run_ours(args):
     import torch.distributed as dist
     from paper_2609_20971_b200 import alloc_stats, rbs_block_stats, rbs_select, rbs_sparse_prefill, workspace_bytes
-    from paper_2609_20971_b200.binding import RBS_OP_SELECT, RbsShape
+    from paper_2609_20971_b200.binding import RBS_OP_SELECT, RBS_OP_SPARSE_PREFILL, RbsShape
     from paper_2609_20971_b200.synth import make_inputs
 
     rank = int(os.environ.get("RANK", "0"))
@@ -368,6 +371,7 @@ def run_ours(args):
     density = torch.empty(L, cfg.Hq, dtype=torch.float32, device=dev)
     shape = RbsShape(L, cfg.N, cfg.Hq, cfg.Hkv, cfg.d, B)
     ws = torch.empty(workspace_bytes(RBS_OP_SELECT, shape), dtype=torch.uint8, device=dev)
+    ws_att = torch.empty(max(256, workspace_bytes(RBS_OP_SPARSE_PREFILL, shape)), dtype=torch.uint8, device=dev)
     sel_args = (cfg.alpha_base, cfg.alpha_rescue, cfg.n_sink, cfg.n_local, cfg.n_recent)
     stream = torch.cuda.current_stream()
 
@@ -443,6 +447,23 @@ def run_ours(args):
     e1.record(stream)
     barrier()
     t_dense = e0.elapsed_time(e1) / n_dense
+
+    # the last 64 query blocks as a chunked call (what a chunked-prefill pipeline issues last): whole rows against rows
+    # of more than 256 key tiles cut into parts (the call is given the schedule's workspace)
+    from paper_2609_20971_b200 import rbs_sparse_prefill_chunk
+    chunk = {}
+    if M > 64 and B >= 128:
+        q0c = M - 64
+        mc, Qc, Oc = mask[:, :, q0c:].contiguous(), Qg[:, q0c * B:], Og[:, q0c * B:]
+        for name, wsa in (("whole_rows", None), ("split_rows", ws_att)):
+            for rep in range(4):
+                if rep == 1:
+                    torch.cuda.synchronize()
+                    e0.record(stream)
+                rbs_sparse_prefill_chunk(Qc, Kg, Vg, mc, B, q0c, out=Oc, workspace=wsa)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            chunk[f"last_64_query_blocks_ms_{name}"] = e0.elapsed_time(e1) / 3
 
     # threshold sweep of the headline config: the paper's three (alpha_base, alpha_rescue) pairs (Sec. 4.4 sensitivity
     # table) and pairs calibrated by bisection to realised densities of about 3 / 5 / 10 / 15 %, timed like the step
@@ -553,6 +574,7 @@ def run_ours(args):
             "stats_clocks": stat_clocks,
             "stats_us_times_sm_mhz": (t_stats_rot * 1e3 * stat_clocks["sm_mhz"]) if stat_clocks and stat_clocks.get("sm_mhz") else None,
             "peaks": peaks,
+            "chunked_call": chunk,
             "sweep": sweep,
             "workloads": others,
             "bench_wall_s": time.time() - T_START,

@@ -236,20 +236,24 @@ def rbs_mask_group_union(mask: torch.Tensor, density: torch.Tensor, n_kv_heads: 
 def rbs_sparse_prefill(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, mask: torch.Tensor | None, block: int, *,
                        out: torch.Tensor | None = None, return_lse: bool = False, softmax_scale: float = 0.0,
                        workspace: torch.Tensor | None = None):
-    """Causal block-sparse attention over `mask` (Sec. 3.3); mask=None is dense causal attention (Eq. 1)."""
+    """Causal block-sparse attention over `mask` (Sec. 3.3); mask=None is dense causal attention (Eq. 1).
+    `workspace` (uint8, at least prefill_workspace_bytes(...)): opt into the row-length-aware schedule (blocks of 128
+    or 256): rows of more than 256 key tiles are cut into parts that run side by side and are merged afterwards."""
     lib = load_library()
     L, N, Hq, d = Q.shape
     shape = RbsShape(L, N, Hq, K.shape[2], d, block)
     if out is None:
         out = torch.empty_like(Q)
     lse = torch.empty(L, Hq, N, dtype=torch.float32, device=Q.device) if return_lse else None
-    need = workspace_bytes(RBS_OP_SPARSE_PREFILL, shape)
-    if workspace is None and need > 0:
-        workspace = torch.empty(need, dtype=torch.uint8, device=Q.device)
     _check(lib.rbs_sparse_prefill(ctypes.byref(shape), _tensor(Q), _tensor(K), _tensor(V), _ptr(mask), _tensor(out),
                                   _ptr(lse), softmax_scale, _ptr(workspace),
                                   0 if workspace is None else workspace.numel(), _stream()), "rbs_sparse_prefill")
     return (out, lse) if return_lse else out
+
+
+def prefill_workspace_bytes(L: int, N: int, Hq: int, Hkv: int, block: int, d: int = 128) -> int:
+    """Bytes of the optional rbs_sparse_prefill / rbs_sparse_prefill_chunk workspace for a sequence of N tokens."""
+    return workspace_bytes(RBS_OP_SPARSE_PREFILL, RbsShape(L, N, Hq, Hkv, d, block))
 
 
 def rbs_select_chunk(Q: torch.Tensor, stats: BlockStats, block: int, seqlen: int, q_start_block: int,
@@ -276,7 +280,7 @@ def rbs_select_chunk(Q: torch.Tensor, stats: BlockStats, block: int, seqlen: int
 
 def rbs_sparse_prefill_chunk(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, mask: torch.Tensor | None, block: int,
                              q_start_block: int, *, out: torch.Tensor | None = None, return_lse: bool = False,
-                             softmax_scale: float = 0.0):
+                             softmax_scale: float = 0.0, workspace: torch.Tensor | None = None):
     """Attention for the query chunk Q [L, Nq, Hq, d] starting at block `q_start_block`, against K, V [L, N, Hkv, d]."""
     lib = load_library()
     L, Nq, Hq, d = Q.shape
@@ -285,6 +289,7 @@ def rbs_sparse_prefill_chunk(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, 
         out = torch.empty_like(Q)
     lse = torch.empty(L, Hq, Nq, dtype=torch.float32, device=Q.device) if return_lse else None
     _check(lib.rbs_sparse_prefill_chunk(ctypes.byref(shape), q_start_block, Nq, _tensor(Q), _tensor(K), _tensor(V),
-                                        _ptr(mask), _tensor(out), _ptr(lse), softmax_scale, None, 0, _stream()),
+                                        _ptr(mask), _tensor(out), _ptr(lse), softmax_scale, _ptr(workspace),
+                                        0 if workspace is None else workspace.numel(), _stream()),
            "rbs_sparse_prefill_chunk")
     return (out, lse) if return_lse else out

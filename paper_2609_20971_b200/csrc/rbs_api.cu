@@ -45,6 +45,22 @@ SelectWorkspace select_workspace(const Dims& x) {
   return w;
 }
 
+// Bounds that hold for every call on a sequence of n_rows query tiles: at most 4 bands, band_rows * bands <= n_rows + 3,
+// 24 extra items, 8 split rows and 32 part slots per (band, batch, KV head) group (the constants of rbs_prefill.cu).
+PrefillWorkspace prefill_workspace(int L, int Hq, int Hkv, int n_rows, int G) {
+  PrefillWorkspace w;
+  const size_t groups = static_cast<size_t>(4) * L * Hkv;
+  const size_t items = static_cast<size_t>(L) * Hkv * (static_cast<size_t>(n_rows) + 4) * G + groups * 24;
+  size_t off = 0;
+  w.off_items = off; off = align_up(off + items * 16, 256);
+  w.off_splits = off; off = align_up(off + groups * 8 * 16, 256);
+  w.off_part_o = off; off = align_up(off + groups * 32 * 128 * 128 * sizeof(float), 256);
+  w.off_part_ml = off; off = align_up(off + groups * 32 * 256 * sizeof(float), 256);
+  w.bytes = off;
+  (void)Hq;
+  return w;
+}
+
 }  // namespace rbs
 
 extern "C" size_t rbs_workspace_bytes(int op, const rbs_shape* shape) {
@@ -52,6 +68,8 @@ extern "C" size_t rbs_workspace_bytes(int op, const rbs_shape* shape) {
   rbs::Dims x = rbs::make_dims(*shape);
   switch (op) {
     case RBS_OP_SELECT: return rbs::select_workspace(x).bytes;
+    case RBS_OP_SPARSE_PREFILL:
+      return x.B >= 128 ? rbs::prefill_workspace(x.L, x.Hq, x.Hkv, x.M * (x.B / 128), x.G).bytes : 0;
     default: return 0;
   }
 }

@@ -47,6 +47,14 @@ struct SelectWorkspace {
 };
 SelectWorkspace select_workspace(const Dims& x);
 
+// Workspace carve-up of rbs_sparse_prefill's row-length-aware schedule (blocks of 128 and 256), sized for the whole
+// sequence so that it also serves every chunked call: the work items, the list of split rows and the partial
+// results of their parts.  n_rows = 128-row query tiles of the sequence.
+struct PrefillWorkspace {
+  size_t off_items, off_splits, off_part_o, off_part_ml, bytes;
+};
+PrefillWorkspace prefill_workspace(int L, int Hq, int Hkv, int n_rows, int G);
+
 // TMA tensor map over a bf16 [L][N][H][d] tensor with arbitrary (16-byte aligned) strides; box = box_d x box_t.
 rbs_status make_tmap_lthd(::CUtensorMap_st* out, const void* ptr, int L, int N, int H, int d, int64_t sb, int64_t st,
                           int64_t sh, int box_d, int box_t, bool swizzle128);

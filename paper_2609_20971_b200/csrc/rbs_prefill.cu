@@ -21,7 +21,22 @@ struct PrefillParams {
   int q0, Mq, Nq;   // this call's queries: first query block (global index), number of blocks, number of tokens
   int band_rows;    // 128-row query tiles per band of the tile order (tensor-core path)
   float scale_log2;
+  // Row-length-aware schedule (null: tiles in their static order, one CTA per tile).  One int4 per CTA:
+  // x = position of the tile in its group's static order (-1: nothing to do), [y, z) = range of 128-key sub-blocks
+  // this item attends, w = slot of its partial result (-1: the item is a whole row and writes O itself).
+  const int4* items;
+  int items_per_group;
+  float* part_o;    // [slot][128 rows][128] unnormalised O of a part, fp32
+  float* part_ml;   // [slot][2][128]        running maximum (log2 units) and row sum of a part
 };
+
+// Rows longer than this many 128-key sub-blocks are cut into parts of equal length that run as separate CTAs and are
+// merged afterwards; the cut depends only on the row itself, so a row is treated the same in every call.
+constexpr int kSplitCap = 256;
+constexpr int kSplitMaxParts = 4;      // parts per split row
+constexpr int kSplitRowsPerGroup = 8;  // split rows per (band, batch, KV head) group: its longest ones
+constexpr int kSplitSlotsPerGroup = kSplitRowsPerGroup * kSplitMaxParts;
+constexpr int kExtraItemsPerGroup = kSplitRowsPerGroup * (kSplitMaxParts - 1);
 
 // next selected key block after `cur` (cur = -1 to start), restricted to b <= i; -1 when exhausted
 __device__ __forceinline__ int next_block(const uint32_t* __restrict__ row, int cur, int i) {
@@ -257,6 +272,7 @@ constexpr float kSumLimit = 16384.0f;
 // 9.89 / 11.32.
 constexpr int kPolyEvery = 16;
 
+template <bool SCHED>
 __global__ void __launch_bounds__(kPfThreads, 2)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                   const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmO,
@@ -285,12 +301,22 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   // The bands keep the very long rows (the dense rows of the last query blocks) of every KV head near the start
   // of the launch: with one band, the last KV head's dense rows started after three quarters of the launch and
   // ran on alone after everything else had finished.
+  // SCHED: the grid follows the item list of plan_rows_kernel instead: the same order, with rows longer than kSplitCap
+  // cut into parts that sit next to each other.
   const int R = p.R;
   const int Hkv = p.Hq / p.G;
-  const int per_band_kv = p.band_rows * p.G;
+  const int per_band_kv = SCHED ? p.items_per_group : p.band_rows * p.G;
   const int per_band = p.L * Hkv * per_band_kv;
   const int band = static_cast<int>(blockIdx.x / per_band), rem_band = static_cast<int>(blockIdx.x % per_band);
-  const int kvid = rem_band / per_band_kv, rem = rem_band % per_band_kv;
+  const int kvid = rem_band / per_band_kv;
+  int rem = rem_band % per_band_kv;
+  // with a schedule the CTA's tile, its range of key sub-blocks and the slot of its partial result come from its item
+  int4 item = make_int4(0, 0, 0x7fffffff, -1);
+  if (SCHED) {
+    item = __ldg(p.items + blockIdx.x);
+    if (item.x < 0) return;                 // unused entry of the group's item list
+    rem = item.x;
+  }
   const int l = kvid / Hkv, hk = kvid % Hkv;
   const int Tl = p.Mq * R - 1 - (band * p.band_rows + rem / p.G);  // 128-row query tile inside this call's chunk
   if (Tl < 0) return;                       // padding of the last band
@@ -299,6 +325,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const int h = hk * p.G + rem % p.G;
   if (Tl * 128 >= p.Nq) return;             // a tile wholly past the end of the queries (short last block of 256)
   const uint32_t* mrow = p.mask ? p.mask + ((static_cast<int64_t>(l) * p.Hq + h) * p.Mq + (i - p.q0)) * p.W : nullptr;
+  const int Tw = SCHED ? min(T, item.z - 1) : T;   // last sub-block this CTA may attend (T itself for a whole row)
+  const int kb0 = SCHED ? item.y - 1 : -1;         // where the walk over the mask row starts
 
   if (tid == 0) {
     mbar_init(smem_u32(&bar_q), 1);
@@ -324,13 +352,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     // ------------------------------- TMA producer -------------------------------
     if (lane == 0) {
       tma_prefetch_desc(&tmQ); tma_prefetch_desc(&tmK); tma_prefetch_desc(&tmV);
-      int b = next_kb(mrow, -1, i, R, T);
+      int b = next_kb(mrow, kb0, i, R, Tw);
       if (b >= 0) {
         mbar_arrive_expect_tx(smem_u32(&bar_q), kTile);
         tma_load_4d(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, Tl * B, l);
         tma_load_4d(smem_u32(sQ + kPanel), &tmQ, smem_u32(&bar_q), 64, h, Tl * B, l);
       }
-      for (int j = 0; b >= 0; ++j, b = next_kb(mrow, b, i, R, T)) {
+      for (int j = 0; b >= 0; ++j, b = next_kb(mrow, b, i, R, Tw)) {
         if (j > 0 && !mbar_wait(smem_u32(&bar_s), (j - 1) & 1, status, kWaitStageFree)) break;   // S_{j-1} done: K free
         mbar_arrive_expect_tx(smem_u32(&bar_kfull), kTile);
         tma_load_4d(smem_u32(sK), &tmK, smem_u32(&bar_kfull), 0, hk, b * B, l);
@@ -348,7 +376,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     // built once (they only differ in the address field) and the next block index is fetched from the
     // mask while the softmax of the current block runs.
     {
-      int b = next_kb(mrow, -1, i, R, T);
+      int b = next_kb(mrow, kb0, i, R, Tw);
       bool ok = b < 0 || mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);
       const uint64_t dq = smem_desc_sw128(smem_u32(sQ), 16, 1024);
       const uint64_t dk = smem_desc_sw128(smem_u32(sK), 16, 1024);
@@ -361,7 +389,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         __syncwarp();
         mma_ss_k128_commit_elect(tmem_s, dq, dk, kIdescQK, kPanel, kPanel, smem_u32(&bar_s));
       };
-      int b_next = b >= 0 ? next_kb(mrow, b, i, R, T) : -1;
+      int b_next = b >= 0 ? next_kb(mrow, b, i, R, Tw) : -1;
       ok = __all_sync(0xffffffffu, ok);
       if (ok && b >= 0) {
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_kfull), 0, status, kWaitTmaFull));
@@ -372,7 +400,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       }
       for (int j = 0; ok && b >= 0; ++j) {
         const uint32_t ph = j & 1;
-        const int b_next2 = b_next >= 0 ? next_kb(mrow, b_next, i, R, T) : -1;   // global-memory latency hidden behind the softmax
+        const int b_next2 = b_next >= 0 ? next_kb(mrow, b_next, i, R, Tw) : -1;   // global-memory latency hidden behind the softmax
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_vfull), ph, status, kWaitTmaFull) &&
                                          mbar_wait(smem_u32(&bar_p), ph, status, kWaitPReady));   // P of keys 0..63
         if (!ok) break;
@@ -397,7 +425,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     const int row = warp * 32 + lane;
     const uint32_t lane_off = static_cast<uint32_t>(warp * 32) << 16;
     float m_used = -INFINITY, l_sum = 0.f;   // m_used in log2 units of the scaled logits
-    int b = next_kb(mrow, -1, i, R, T);
+    int b = next_kb(mrow, kb0, i, R, Tw);
     const bool any_block = b >= 0;
     bool ok = true;
     int j = 0;
@@ -515,6 +543,27 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         for (int c = 0; c < 16; ++c) reinterpret_cast<uint4*>(orow)[c] = make_uint4(0, 0, 0, 0);
         if (lse_dst) *lse_dst = -INFINITY;
       }
+    } else if (SCHED && __ldg(&p.items[blockIdx.x].w) >= 0) {
+      const int part_slot = __ldg(&p.items[blockIdx.x].w);   // (read again here rather than kept in a register all along)
+      // a part of a split row: the unnormalised O row, the maximum in use and the row sum go to the part's slot;
+      // combine_parts_kernel merges the parts of the row in a fixed order
+      const bool o_ready = __all_sync(0xffffffffu, ok && mbar_wait(smem_u32(&bar_pv), (j - 1) & 1, status, kWaitOReady));
+      tc_fence_after_sync();
+      float* po = p.part_o + (static_cast<int64_t>(part_slot) * 128 + row) * 128;
+#pragma unroll 1
+      for (int c0 = 0; o_ready && c0 < 128; c0 += 32) {
+        uint32_t r[32];
+        tmem_ld32(tmem_o + lane_off + c0, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int q = 0; q < 32; q += 4)
+          *reinterpret_cast<uint4*>(po + c0 + q) = make_uint4(r[q], r[q + 1], r[q + 2], r[q + 3]);
+      }
+      if (o_ready) {
+        float* ml = p.part_ml + static_cast<int64_t>(part_slot) * 256;
+        ml[row] = m_used;
+        ml[128 + row] = l_sum;
+      }
     } else {
       // every thread of the four warps reaches the barrier below, also one whose wait has given up
       const bool o_ready = __all_sync(0xffffffffu, ok && mbar_wait(smem_u32(&bar_pv), (j - 1) & 1, status, kWaitOReady));
@@ -558,8 +607,181 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   if (warp == 5) tmem_dealloc(s_tmem, 256);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Row-length-aware schedule of prefill_tc_kernel (the index compaction of the method's complexity paragraph, Sec. 3.3,
+// in the form this kernel needs: per-row counts of selected blocks, long rows cut into parts).
+// One CTA per group = (band of query tiles, batch, KV head), the unit inside which the static order keeps the K/V of
+// one KV head in flight.  It counts the selected 128-key sub-blocks of each of the group's rows from the mask and
+// writes one item per CTA of the attention kernel, in the static order (rows from the end of the sequence backwards,
+// i.e. longest candidate range first, the G heads of a row together).  The first kSplitRowsPerGroup rows of that
+// order that exceed kSplitCap sub-blocks are cut into up to kSplitMaxParts parts of equal length, placed next to each
+// other.  (Sorting the rows of a group by their counts was measured as well: 0.03 - 0.1 ms slower on the 128K layer.)
+// ---------------------------------------------------------------------------------------------
+constexpr int kPlanThreads = 1024;
+
+// number of 128-key sub-blocks tile T of query block i attends in mask row `row`: R per selected block below the
+// diagonal block, and the diagonal block's sub-blocks up to T
+__device__ __forceinline__ int count_kb_fast(const uint32_t* __restrict__ row, int i, int R, int T) {
+  int n = 0;
+  const int wi = i >> 5;
+  for (int w = 0; w < wi; ++w) n += __popc(__ldg(row + w));
+  const uint32_t u = __ldg(row + wi) & (0xffffffffu >> (31 - (i & 31)));
+  const uint32_t diag = (u >> (i & 31)) & 1u;
+  return R * (n + __popc(u) - static_cast<int>(diag)) + (diag ? T - i * R + 1 : 0);
+}
+
+// the same count by walking the set bits, stopping at ordinal `stop` (>= 0): *kb_at receives the index of the
+// sub-block with that ordinal
+__device__ __forceinline__ int count_kb(const uint32_t* __restrict__ row, int i, int R, int T, int stop, int* kb_at) {
+  int n = 0;
+  for (int w = 0; w <= (i >> 5); ++w) {
+    uint32_t u = __ldg(row + w);
+    if (((w + 1) << 5) - 1 > i) u &= 0xffffffffu >> (31 - (i & 31));
+    while (u) {
+      const int b = (w << 5) + __ffs(u) - 1;
+      u &= u - 1;
+      const int first = b * R, last = min(b * R + R - 1, T);   // this block's sub-blocks up to the diagonal
+      if (stop >= 0 && n + (last - first + 1) > stop) { *kb_at = first + (stop - n); return stop; }
+      n += last - first + 1;
+    }
+  }
+  return n;
+}
+
+__global__ void __launch_bounds__(kPlanThreads)
+plan_rows_kernel(const PrefillParams p, int4* __restrict__ items, int4* __restrict__ splits) {
+  extern __shared__ int s_cnt[];                     // sub-blocks per row of the group, in static order
+  __shared__ int s_warp_long[kPlanThreads / 32];
+  __shared__ int s_split_pos[kSplitRowsPerGroup], s_split_parts[kSplitRowsPerGroup], s_n_split;
+  const int R = p.R, Hkv = p.Hq / p.G;
+  const int n_g = p.band_rows * p.G;               // rows (128-row tiles) per group
+  const int g = blockIdx.x;                        // band * (L * Hkv) + kvid
+  const int band = g / (p.L * Hkv), kvid = g % (p.L * Hkv);
+  const int l = kvid / Hkv, hk = kvid % Hkv;
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  auto tile_of = [&](int pos, int& Tl, int& T, int& i, const uint32_t*& row) -> bool {
+    Tl = p.Mq * R - 1 - (band * p.band_rows + pos / p.G);
+    if (Tl < 0 || Tl * 128 >= p.Nq) return false;
+    T = p.q0 * R + Tl;
+    i = T / R;
+    const int h = hk * p.G + pos % p.G;
+    row = p.mask + ((static_cast<int64_t>(l) * p.Hq + h) * p.Mq + (i - p.q0)) * p.W;
+    return true;
+  };
+  // every thread owns a contiguous run of rows, so that ranks in static order come from one scan over the threads
+  const int per_thread = (n_g + kPlanThreads - 1) / kPlanThreads;
+  const int first = tid * per_thread, last = min(n_g, first + per_thread);
+  int n_long = 0;
+  for (int pos = first; pos < last; ++pos) {
+    int Tl, T, i;
+    const uint32_t* row;
+    const int cnt = tile_of(pos, Tl, T, i, row) ? count_kb_fast(row, i, R, T) : -1;   // -1: no such tile
+    s_cnt[pos] = cnt;
+    n_long += cnt > kSplitCap;
+  }
+  if (tid == 0) s_n_split = 0;
+  // exclusive scan of n_long over the threads
+  int incl = n_long;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const int v = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += v;
+  }
+  if (lane == 31) s_warp_long[warp] = incl;
+  __syncthreads();
+  int rank = incl - n_long;
+  for (int w = 0; w < warp; ++w) rank += s_warp_long[w];
+  for (int pos = first; pos < last && rank < kSplitRowsPerGroup; ++pos) {
+    const int cnt = s_cnt[pos];
+    if (cnt > kSplitCap) {
+      s_split_pos[rank] = pos;
+      s_split_parts[rank] = min(kSplitMaxParts, (cnt + kSplitCap - 1) / kSplitCap);
+      atomicMax(&s_n_split, rank + 1);
+      ++rank;
+    }
+  }
+  __syncthreads();
+  const int n_split = s_n_split;
+  const int per_group = n_g + kExtraItemsPerGroup;
+  int4* out = items + static_cast<int64_t>(g) * per_group;
+  int extra_total = 0;
+  for (int s = 0; s < n_split; ++s) extra_total += s_split_parts[s] - 1;
+  // whole rows
+  for (int pos = first; pos < last; ++pos) {
+    int at = pos;
+    bool is_split = false;
+    for (int s = 0; s < n_split; ++s) {
+      if (s_split_pos[s] < pos) at += s_split_parts[s] - 1;
+      is_split |= s_split_pos[s] == pos;
+    }
+    if (!is_split) out[at] = s_cnt[pos] >= 0 ? make_int4(pos, 0, 0x7fffffff, -1) : make_int4(-1, 0, 0, -1);
+  }
+  for (int e = n_g + extra_total + tid; e < per_group; e += kPlanThreads) out[e] = make_int4(-1, 0, 0, -1);   // unused
+  // the parts of the split rows: one thread per (row, part)
+  if (tid < kSplitRowsPerGroup * kSplitMaxParts) {
+    const int s = tid / kSplitMaxParts, part = tid % kSplitMaxParts;
+    if (s < n_split) {
+      const int pos = s_split_pos[s], parts = s_split_parts[s], cnt = s_cnt[pos];
+      if (part < parts) {
+        int at = pos + part;
+        for (int s2 = 0; s2 < s; ++s2) at += s_split_parts[s2] - 1;
+        int Tl, T, i;
+        const uint32_t* row;
+        tile_of(pos, Tl, T, i, row);
+        const int len = (cnt + parts - 1) / parts;
+        int kb_begin = 0, kb_end = T + 1;
+        if (part > 0) count_kb(row, i, R, T, part * len, &kb_begin);
+        if (part + 1 < parts) count_kb(row, i, R, T, (part + 1) * len, &kb_end);
+        out[at] = make_int4(pos, kb_begin, kb_end, g * kSplitSlotsPerGroup + s * kSplitMaxParts + part);
+      }
+      if (part == 0) splits[g * kSplitRowsPerGroup + s] = make_int4(pos, parts, 0, 0);
+    } else if (part == 0) {
+      splits[g * kSplitRowsPerGroup + s] = make_int4(-1, 1, 0, 0);
+    }
+  }
+}
+
+// Merges the parts of one split row: with m = max_p m_p,  l = sum_p l_p 2^(m_p - m),  O = sum_p O_p 2^(m_p - m) / l
+// (the maximum is only a shift, Sec. 3.3's softmax over the retained keys is unchanged), parts taken in order.
+// One CTA per (group, split-row slot), one thread per query row.
+__global__ void __launch_bounds__(128)
+combine_parts_kernel(const PrefillParams p, const int4* __restrict__ splits) {
+  const int4 sp = splits[blockIdx.x];
+  if (sp.x < 0) return;
+  const int g = blockIdx.x / kSplitRowsPerGroup, s = blockIdx.x % kSplitRowsPerGroup;
+  const int R = p.R, Hkv = p.Hq / p.G;
+  const int band = g / (p.L * Hkv), kvid = g % (p.L * Hkv);
+  const int l = kvid / Hkv, hk = kvid % Hkv;
+  const int Tl = p.Mq * R - 1 - (band * p.band_rows + sp.x / p.G);
+  const int h = hk * p.G + sp.x % p.G;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int slot0 = g * kSplitSlotsPerGroup + s * kSplitMaxParts;
+  // a warp takes one query row at a time, its lanes four output columns each (whole 512-byte lines per part)
+  for (int row = warp; row < 128; row += 4) {
+    if (Tl * 128 + row >= p.Nq) break;     // rows past the end of the queries are not written
+    float m = -INFINITY;
+    for (int q = 0; q < sp.y; ++q) m = fmaxf(m, p.part_ml[static_cast<int64_t>(slot0 + q) * 256 + row]);
+    float lsum = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int q = 0; q < sp.y; ++q) {
+      const float* ml = p.part_ml + static_cast<int64_t>(slot0 + q) * 256;
+      const float w = fast_exp2(ml[row] - m);
+      lsum = fmaf(ml[128 + row], w, lsum);
+      const float4 a = *reinterpret_cast<const float4*>(p.part_o + (static_cast<int64_t>(slot0 + q) * 128 + row) * 128 + lane * 4);
+      acc.x = fmaf(a.x, w, acc.x); acc.y = fmaf(a.y, w, acc.y); acc.z = fmaf(a.z, w, acc.z); acc.w = fmaf(a.w, w, acc.w);
+    }
+    const float inv = 1.0f / lsum;
+    __nv_bfloat16* orow = p.O + l * p.osb + (static_cast<int64_t>(Tl) * 128 + row) * p.ost + h * p.osh;
+    uint2 v;
+    v.x = pack_bf16(acc.x * inv, acc.y * inv);
+    v.y = pack_bf16(acc.z * inv, acc.w * inv);
+    *reinterpret_cast<uint2*>(orow + lane * 4) = v;
+    if (p.lse && lane == 0) p.lse[(static_cast<int64_t>(l) * p.Hq + h) * p.Nq + Tl * 128 + row] = (m + fast_log2(lsum)) * 0.6931471805599453f;
+  }
+}
+
 static rbs_status launch_prefill_tc(const PrefillParams& p, const rbs_tensor& Q, const rbs_tensor& K,
-                                    const rbs_tensor& V, int Hkv, cudaStream_t s) {
+                                    const rbs_tensor& V, int Hkv, void* workspace, size_t workspace_bytes, cudaStream_t s) {
   CUtensorMap tmQ, tmK, tmV;
   rbs_status st;
   if ((st = make_tmap_lthd(&tmQ, Q.ptr, p.L, p.Nq, p.Hq, kHeadDim, Q.stride_batch, Q.stride_token, Q.stride_head, 64, 128, true)) != RBS_OK) return st;
@@ -571,7 +793,8 @@ static rbs_status launch_prefill_tc(const PrefillParams& p, const rbs_tensor& Q,
   unsigned int* status = device_status_ptr();
   if (status == nullptr) return RBS_ERR_CUDA;
   const size_t smem = 3 * 2 * 128 * 128;
-  if ((st = ensure_dynamic_smem(reinterpret_cast<const void*>(prefill_tc_kernel), smem)) != RBS_OK) return st;
+  if ((st = ensure_dynamic_smem(reinterpret_cast<const void*>(prefill_tc_kernel<false>), smem)) != RBS_OK) return st;
+  if ((st = ensure_dynamic_smem(reinterpret_cast<const void*>(prefill_tc_kernel<true>), smem)) != RBS_OK) return st;
   PrefillParams pp = p;
   const int n_rows = p.Mq * p.R;
   // up to four bands of at least 64 query tiles (512 CTAs per band and KV head at G = 8: enough to fill the GPU
@@ -580,10 +803,37 @@ static rbs_status launch_prefill_tc(const PrefillParams& p, const rbs_tensor& Q,
   int n_bands = n_rows / 64;
   n_bands = n_bands < 1 ? 1 : (n_bands > 4 ? 4 : n_bands);
   pp.band_rows = (n_rows + n_bands - 1) / n_bands;
-  const long long n_cta = static_cast<long long>(p.L) * p.Hq * pp.band_rows * n_bands;
+  const int n_groups = n_bands * p.L * Hkv;
+  const int rows_per_group = pp.band_rows * p.G;
+  pp.items = nullptr; pp.items_per_group = 0; pp.part_o = nullptr; pp.part_ml = nullptr;
+  int4* splits = nullptr;
+  // the schedule needs the mask (dense attention keeps one CTA per tile: its launch is long and its rows shrink
+  // steadily) and a group whose counts fit the planner's shared memory
+  const size_t plan_smem = static_cast<size_t>(rows_per_group) * sizeof(int);
+  const bool scheduled = p.mask != nullptr && workspace != nullptr && plan_smem <= 200 * 1024;
+  if (scheduled) {
+    const PrefillWorkspace w = prefill_workspace(p.L, p.Hq, Hkv, p.M * p.R, p.G);
+    if (workspace_bytes < w.bytes || reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return RBS_ERR_WORKSPACE;
+    unsigned char* base = static_cast<unsigned char*>(workspace);
+    int4* items = reinterpret_cast<int4*>(base + w.off_items);
+    splits = reinterpret_cast<int4*>(base + w.off_splits);
+    pp.items = items;
+    pp.items_per_group = rows_per_group + kExtraItemsPerGroup;
+    pp.part_o = reinterpret_cast<float*>(base + w.off_part_o);
+    pp.part_ml = reinterpret_cast<float*>(base + w.off_part_ml);
+    if ((st = ensure_dynamic_smem(reinterpret_cast<const void*>(plan_rows_kernel), plan_smem)) != RBS_OK) return st;
+    plan_rows_kernel<<<n_groups, kPlanThreads, plan_smem, s>>>(pp, items, splits);
+    RBS_CUDA_OK(cudaGetLastError());
+  }
+  const long long n_cta = static_cast<long long>(n_groups) * (scheduled ? pp.items_per_group : rows_per_group);
   if (n_cta > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
-  prefill_tc_kernel<<<static_cast<unsigned>(n_cta), kPfThreads, smem, s>>>(tmQ, tmK, tmV, tmO, pp, status);
+  if (scheduled) prefill_tc_kernel<true><<<static_cast<unsigned>(n_cta), kPfThreads, smem, s>>>(tmQ, tmK, tmV, tmO, pp, status);
+  else prefill_tc_kernel<false><<<static_cast<unsigned>(n_cta), kPfThreads, smem, s>>>(tmQ, tmK, tmV, tmO, pp, status);
   RBS_CUDA_OK(cudaGetLastError());
+  if (scheduled) {
+    combine_parts_kernel<<<n_groups * kSplitRowsPerGroup, 128, 0, s>>>(pp, splits);
+    RBS_CUDA_OK(cudaGetLastError());
+  }
   return RBS_OK;
 }
 
@@ -954,7 +1204,6 @@ static rbs_status prefill_impl(const rbs_shape* shape, int q_start_block, int n_
                                rbs_tensor V, const uint32_t* mask, rbs_tensor O, float* lse, float softmax_scale,
                                void* workspace, size_t workspace_bytes, void* stream) {
   using namespace rbs;
-  (void)workspace; (void)workspace_bytes;
   rbs_status st = check_shape(shape);
   if (st != RBS_OK) return st;
   if ((st = check_tensor(Q)) != RBS_OK || (st = check_tensor(K)) != RBS_OK || (st = check_tensor(V)) != RBS_OK ||
@@ -976,7 +1225,11 @@ static rbs_status prefill_impl(const rbs_shape* shape, int q_start_block, int n_
   p.scale_log2 = scale * kLog2e;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   p.R = x.B / 128;
-  if (x.B >= 128) return launch_prefill_tc(p, Q, K, V, x.Hkv, s);   // tensor-core path (blocks of 128 or 256)
+  if (x.B >= 128 && mask != nullptr && workspace != nullptr) {   // checked before anything touches the GPU
+    const PrefillWorkspace w = prefill_workspace(x.L, x.Hq, x.Hkv, x.M * p.R, x.G);
+    if (workspace_bytes < w.bytes || reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return RBS_ERR_WORKSPACE;
+  }
+  if (x.B >= 128) return launch_prefill_tc(p, Q, K, V, x.Hkv, workspace, workspace_bytes, s);   // tensor-core path (blocks of 128 or 256)
   if (mask == nullptr && (q_start_block & 1) == 0) {
     // Dense attention does not depend on the block size: blocks of 64 run on the tensor-core path as blocks of 128
     // (a chunk has to start on a 128-token boundary for that).
@@ -985,7 +1238,7 @@ static rbs_status prefill_impl(const rbs_shape* shape, int q_start_block, int n_
     p.Mq = (n_q_tokens + 127) / 128;
     p.M = (x.N + 127) / 128;
     p.W = (p.M + 31) / 32;
-    return launch_prefill_tc(p, Q, K, V, x.Hkv, s);
+    return launch_prefill_tc(p, Q, K, V, x.Hkv, nullptr, 0, s);
   }
   if (mask != nullptr) return launch_prefill_tc64(p, Q, K, V, x.Hkv, s);   // blocks of 64, two query blocks per tile
   return launch_prefill<64>(p, s);   // dense chunk from an odd block of 64: register-softmax mma.sync kernel

@@ -10,7 +10,7 @@ from __future__ import annotations
 
 import torch
 
-from .binding import (RBS_OP_SELECT, RbsShape, alloc_stats, rbs_block_stats, rbs_select_chunk, rbs_sparse_prefill_chunk,
+from .binding import (RBS_OP_SELECT, RBS_OP_SPARSE_PREFILL, RbsShape, alloc_stats, rbs_block_stats, rbs_select_chunk, rbs_sparse_prefill_chunk,
                       workspace_bytes)
 
 
@@ -37,6 +37,7 @@ class HostPrefill:
         self.density = torch.empty(n_chunks, L, Hq, dtype=torch.float32, device=self.dev)
         shape = RbsShape(L, N, Hq, Hkv, d, block)
         self.ws = torch.empty(max(256, workspace_bytes(RBS_OP_SELECT, shape)), dtype=torch.uint8, device=self.dev)
+        self.ws_att = torch.empty(max(256, workspace_bytes(RBS_OP_SPARSE_PREFILL, shape)), dtype=torch.uint8, device=self.dev)
         self.s_in, self.s_out = torch.cuda.Stream(self.dev), torch.cuda.Stream(self.dev)
 
     def chunks(self):
@@ -70,7 +71,8 @@ class HostPrefill:
             mc = self.masks[c]
             rbs_select_chunk(self.Qg[:, t0:t1], self.stats, self.B, self.N, q0, alpha_base, alpha_rescue, n_sink, n_local,
                              n_recent, mask=mc, density=self.density[c], workspace=self.ws)
-            rbs_sparse_prefill_chunk(self.Qg[:, t0:t1], self.Kg, self.Vg, mc, self.B, q0, out=self.Og[:, t0:t1])
+            rbs_sparse_prefill_chunk(self.Qg[:, t0:t1], self.Kg, self.Vg, mc, self.B, q0, out=self.Og[:, t0:t1],
+                                     workspace=self.ws_att)
             o_ready = torch.cuda.Event()
             o_ready.record(main)
             with torch.cuda.stream(self.s_out):
@@ -130,7 +132,7 @@ def prefill_varlen(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, cu_seqlens
             rbs_sparse_prefill(q, kk, v, mask, block, out=o)
             densities.append(dens)
             for t in (stats.centroid, stats.radius, stats.beta, stats.rq, mask, dens):
-                t.record_stream(s)
+                t.record_stream(s)       # (the calls' own workspaces are torch allocations made under stream s)
     for s in streams:
         if s != cur:
             cur.wait_stream(s)

@@ -83,7 +83,6 @@ def test_select_argument_checks(lib):
     assert call(alpha_r=-1.0) == INVALID
     assert call(sink=-1) == INVALID
     assert call(mask=None) == INVALID
-    assert call(ws=None) == WORKSPACE
     assert call(ws_bytes=need - 1) == WORKSPACE
     assert call(ws=ctypes.c_void_p(0x1010)) == WORKSPACE          # not 256-byte aligned
 
@@ -92,6 +91,19 @@ def test_prefill_argument_checks(lib):
     good = RbsShape(1, 1024, 4, 2, 128, 128)
     assert lib.rbs_sparse_prefill(ctypes.byref(good), _t(), _t(), _t(ptr=0), None, _t(), None, 0.0, None, 0, None) == INVALID
     assert lib.rbs_sparse_prefill(ctypes.byref(good), _t(), _t(), _t(), None, _t(), None, -1.0, None, 0, None) == INVALID
+
+
+def test_prefill_workspace_checks(lib):
+    good = RbsShape(1, 4096, 4, 2, 128, 128)
+    need = lib.rbs_workspace_bytes(2, ctypes.byref(good))
+    assert need > 0 and need % 256 == 0
+    assert lib.rbs_workspace_bytes(2, ctypes.byref(RbsShape(1, 4096, 4, 2, 128, 64))) == 0   # blocks of 64: no schedule
+    p = ctypes.c_void_p(0x1000)
+
+    def call(mask=p, ws=p, ws_bytes=need):
+        return lib.rbs_sparse_prefill(ctypes.byref(good), _t(), _t(), _t(), mask, _t(), None, 0.0, ws, ws_bytes, None)
+    assert call(ws_bytes=need - 1) == WORKSPACE
+    assert call(ws=ctypes.c_void_p(0x1010)) == WORKSPACE
 
 
 def test_binding_fails_loudly_when_library_is_missing(monkeypatch, tmp_path):

@@ -495,3 +495,42 @@ def test_batch_stride_beyond_32_bits():
     assert torch.equal(mask_v, mask) and torch.equal(dens_v, dens)
     assert torch.equal(Ov, O)
     assert not torch.equal(O[0], O[1])               # the two layers really differ
+
+
+@pytest.mark.parametrize("B,M,tail", [(128, 300, 77), (256, 140, 0)])
+def test_long_rows_are_split_and_merged(B, M, tail):
+    """Rows of more than 256 key tiles of 128 are cut into parts that run as separate CTAs and are merged afterwards
+    (here the dense "recent" rows and a hand-made long row): outputs and lse against the oracle, bit-identical results
+    when the same rows are computed by chunked calls, and a second launch gives the same bits."""
+    from paper_2609_20971_b200 import rbs_sparse_prefill_chunk
+    cfg = SynthConfig("split", N=B * (M - 1) + (tail or B), Hq=4, Hkv=2, B=B, sigma=(0.1, 1.0), seed=61, n_recent=2)
+    Q, K, V = make_inputs(cfg)
+    dev = torch.device("cuda:0")
+    Qg, Kg, Vg = Q.to(dev), K.to(dev), V.to(dev)
+    stats = rbs_block_stats(Kg, B)
+    mask, _ = rbs_select(Qg, stats, B, cfg.alpha_base, cfg.alpha_rescue, 1, 1, cfg.n_recent)
+    dense = unpack_mask(mask, cfg.M)
+    dense[0, 1, cfg.M - 5, : cfg.M - 4] = True          # one more long row, not at the end, for one head only
+    dense[0, 1, cfg.M - 5, 3:40:2] = False              # with holes
+    mask = pack_mask(dense).to(dev)
+    from paper_2609_20971_b200.binding import prefill_workspace_bytes
+    ws = torch.empty(prefill_workspace_bytes(1, cfg.N, cfg.Hq, cfg.Hkv, B), dtype=torch.uint8, device=dev)
+    O, lse = rbs_sparse_prefill(Qg, Kg, Vg, mask, B, return_lse=True, workspace=ws)
+    O2 = rbs_sparse_prefill(Qg, Kg, Vg, mask, B, workspace=ws)
+    O_plain = rbs_sparse_prefill(Qg, Kg, Vg, mask, B)          # no workspace: every row whole
+    torch.cuda.synchronize()
+    assert torch.equal(O, O2)
+    assert (O.float() - O_plain.float()).abs().max().item() <= OUT_MAX_ABS
+    short = slice(0, 200 * 128)                                  # rows that are not cut give the same bits either way
+    assert torch.equal(O[:, short], O_plain[:, short])
+    Q64, K64, V64 = to_f64(Q), to_f64(K), to_f64(V)
+    for h, i in ((0, cfg.M - 1), (3, cfg.M - 2), (1, cfg.M - 5), (1, cfg.M - 6), (2, 5)):
+        ref, lref = orc.masked_attention_block(Q64[0, :, h], K64[0, :, h // 2], V64[0, :, h // 2], dense[0, h, i], i, B)
+        t0, t1 = i * B, min(cfg.N, (i + 1) * B)
+        _check_output(O[0, t0:t1, h].float().cpu().numpy(), ref)
+        assert np.allclose(lse[0, h, t0:t1].cpu().numpy(), lref, atol=2e-3, rtol=1e-4)
+    # the last query blocks again as a chunk of their own: the same rows are cut the same way
+    q0 = cfg.M - 7
+    oc, lc = rbs_sparse_prefill_chunk(Qg[:, q0 * B:], Kg, Vg, mask[:, :, q0:].contiguous(), B, q0, return_lse=True,
+                                      workspace=ws)
+    assert torch.equal(oc, O[:, q0 * B:]) and torch.equal(lc, lse[:, :, q0 * B:])
