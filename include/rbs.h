@@ -72,7 +72,14 @@ typedef struct {
   float* rq;       /* [L][Hkv][2]     (r_low, r_high) = radius quantiles 0.5 and 0.9 */
 } rbs_stats;
 
-enum { RBS_OP_BLOCK_STATS = 0, RBS_OP_SELECT = 1, RBS_OP_SPARSE_PREFILL = 2 };
+/* Per-block coordinate-wise key minima and maxima (App. D.2: a_b, u_b), device fp32, the statistics of the Quest-style
+ * comparison selector. */
+typedef struct {
+  float* lo; /* [L][Hkv][M][d]  a_bj = min over the block's keys of k_j */
+  float* hi; /* [L][Hkv][M][d]  u_bj = max over the block's keys of k_j */
+} rbs_box;
+
+enum { RBS_OP_BLOCK_STATS = 0, RBS_OP_SELECT = 1, RBS_OP_SPARSE_PREFILL = 2, RBS_OP_SELECT_BOX = 3 };
 
 /* Bytes of device workspace the given call needs for this shape (0 if none).  Workspace must be
  * 256-byte aligned; its contents need not be initialised and are undefined afterwards. */
@@ -176,6 +183,26 @@ RBS_API rbs_status rbs_select_variant(const rbs_shape* shape, rbs_tensor Q, rbs_
                                       uint32_t* mask, float* density, uint32_t* dbg_base_mask,
                                       uint32_t* dbg_rescue_mask, void* workspace, size_t workspace_bytes,
                                       void* stream);
+
+/*
+ * The Quest-style comparison selector of the paper's ablation (Sec. 4.2; App. D.2, Eq. quest_box), in the same backend.
+ *   rbs_block_stats_box  as rbs_block_stats, and from the same single read of K also box.lo / box.hi: the
+ *                        per-coordinate minimum and maximum of each block's keys.
+ *   rbs_select_box       block logit = the box upper bound  U_b(q) = sum_j max(q_j a_bj, q_j u_bj) = q.v_b + |q|.h_b
+ *                        (v_b, h_b the box centre and half-width), aggregated over the query block's tokens exactly as the
+ *                        other selectors' logits are (Eq. block_aggregation); query block i then keeps its
+ *                        ceil(density_param * (i + 1)) best causal key blocks -- blocks whose score equals the last kept
+ *                        one included -- united with the forced blocks of rbs_select.
+ * The paper states the policy only as "per-dimension key minima/maxima and query-dependent block selection" with a
+ * "density parameter" (0.0405 in its comparison); aggregation and the meaning of the parameter are this library's
+ * reading.  mask, density: as rbs_select.  dbg_chosen_mask (nullable): the choice before the union with the forced
+ * blocks.  Blocks of 64 and 128 only (RBS_ERR_UNSUPPORTED for 256).  density_param in (0, 1].
+ * Workspace: rbs_workspace_bytes(RBS_OP_SELECT_BOX, shape).
+ */
+RBS_API rbs_status rbs_block_stats_box(const rbs_shape* shape, rbs_tensor K, rbs_stats stats, rbs_box box, void* stream);
+RBS_API rbs_status rbs_select_box(const rbs_shape* shape, rbs_tensor Q, rbs_box box, double density_param, int n_sink,
+                                  int n_local, int n_recent, uint32_t* mask, float* density, uint32_t* dbg_chosen_mask,
+                                  void* workspace, size_t workspace_bytes, void* stream);
 
 /*
  * rbs_select for callers that have no device memory to hand over and must not allocate any.

@@ -29,6 +29,15 @@ causal attention == a library attention routine, invariances (shift, rotation, m
 alpha).  Parity unpinned (a reading only; nothing in the paper fixes them): the quantile
 interpolation rule, per-query-head mask granularity under GQA, the meaning and units of
 sink/local/recent, and scoring of the diagonal block.
+
+The Quest-style comparison selector (Sec. 4.2; App. D.2, Eq. quest_box) is restated too: per-coordinate
+minima / maxima per block (box_stats), the box upper bound as the block logit (box_logits; pinned by
+the App. D.2 values and by "bound >= every token logit"), and block selection by a density parameter.
+The paper only says the adaptation "uses per-dimension key minima/maxima and query-dependent block
+selection" with "density parameter 0.0405" in "a shared prefill backend".  Reading taken, PARITY
+UNPINNED: the box logit goes through the same aggregation over the query block's tokens as the
+other selectors (Eq. block_aggregation); query block i keeps its ceil(delta * (i + 1)) best causal
+blocks, ties with the last kept score included, united with the same forced blocks.
 """
 from __future__ import annotations
 
@@ -280,6 +289,74 @@ def box_upper_bound(q: np.ndarray, keys: np.ndarray) -> float:
     a = keys.min(axis=0)
     u = keys.max(axis=0)
     return float(np.maximum(q * a, q * u).sum())
+
+
+# --------------------------------------------------------------------------------------
+# Sec. 4.2 / App. D.2: the Quest-style comparison selector
+# --------------------------------------------------------------------------------------
+def box_stats(K: np.ndarray, block: int):
+    """a_b = per-coordinate minimum, u_b = per-coordinate maximum of the block's keys (App. D.2).
+    K [N, d] of one KV head.  Returns (lo [M, d], hi [M, d])."""
+    K = np.asarray(K, dtype=np.float64)
+    N, d = K.shape
+    M = n_blocks(N, block)
+    lo = np.zeros((M, d))
+    hi = np.zeros((M, d))
+    for b in range(M):
+        keys = K[b * block:min(N, (b + 1) * block)]
+        lo[b] = keys.min(axis=0)
+        hi[b] = keys.max(axis=0)
+    return lo, hi
+
+
+def box_logits(Qi: np.ndarray, lo: np.ndarray, hi: np.ndarray) -> np.ndarray:
+    """U_b^box(q) = sum_j max(q_j a_bj, q_j u_bj) for every token of Qi [T, d] and block (Eq. quest_box),
+    coordinate by coordinate as printed.  Returns [T, nb]."""
+    Qi = np.asarray(Qi, dtype=np.float64)
+    out = np.zeros((Qi.shape[0], lo.shape[0]))
+    for b in range(lo.shape[0]):
+        out[:, b] = np.maximum(Qi * lo[b][None, :], Qi * hi[b][None, :]).sum(axis=1)
+    return out
+
+
+def top_fraction(S: np.ndarray, delta: float) -> np.ndarray:
+    """Keeps the ceil(delta * n) largest of the n scores; scores equal to the last kept one are kept too."""
+    n = S.shape[0]
+    k = min(n, max(1, int(math.ceil(delta * n))))
+    kth = np.sort(S)[n - k]
+    return S >= kth
+
+
+@dataclass
+class BoxSelection:
+    chosen: np.ndarray    # [M, M] bool: the density-parameter choice alone
+    forced: np.ndarray    # [M, M] bool
+    final: np.ndarray     # [M, M] bool = chosen | forced
+    margin: np.ndarray    # [M, M] |S - S_kth| / S_kth, the k-th largest score of the row; +inf above the diagonal
+    density: float
+
+
+def select_head_box(Q: np.ndarray, lo: np.ndarray, hi: np.ndarray, block: int, delta: float,
+                    n_sink: int, n_local: int, n_recent: int, rows=None) -> BoxSelection:
+    """Quest-style selection for ONE query head against its KV head's boxes (see the module header for the
+    reading): S_{i,b} = sum_t exp(U_b^box(q_t)/sqrt(d) - m_i), keep the ceil(delta (i + 1)) best b <= i."""
+    Q = np.asarray(Q, dtype=np.float64)
+    N, d = Q.shape
+    M = n_blocks(N, block)
+    chosen = np.zeros((M, M), dtype=bool)
+    forced = np.zeros((M, M), dtype=bool)
+    margin = np.full((M, M), np.inf)
+    for i in (range(M) if rows is None else rows):
+        Qi = Q[i * block:min(N, (i + 1) * block)]
+        nb = i + 1
+        S = aggregate(box_logits(Qi, lo[:nb], hi[:nb]), d)
+        chosen[i, :nb] = top_fraction(S, delta)
+        forced[i, :nb] = forced_blocks(i, M, n_sink, n_local, n_recent)
+        k = min(nb, max(1, int(math.ceil(delta * nb))))
+        kth = np.sort(S)[nb - k]
+        margin[i, :nb] = np.abs(S - kth) / kth
+    final = chosen | forced
+    return BoxSelection(chosen, forced, final, margin, density(final))
 
 
 # --------------------------------------------------------------------------------------

@@ -15,7 +15,7 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "librbs_b200.so")
 
-RBS_OP_BLOCK_STATS, RBS_OP_SELECT, RBS_OP_SPARSE_PREFILL = 0, 1, 2
+RBS_OP_BLOCK_STATS, RBS_OP_SELECT, RBS_OP_SPARSE_PREFILL, RBS_OP_SELECT_BOX = 0, 1, 2, 3
 SELECTOR_RBS, SELECTOR_CENTROID_ONLY, SELECTOR_FULL_L2 = 0, 1, 2
 
 
@@ -32,6 +32,10 @@ class RbsTensor(ctypes.Structure):
 class RbsStats(ctypes.Structure):
     _fields_ = [("centroid", ctypes.c_void_p), ("radius", ctypes.c_void_p),
                 ("beta", ctypes.c_void_p), ("rq", ctypes.c_void_p)]
+
+
+class RbsBox(ctypes.Structure):
+    _fields_ = [("lo", ctypes.c_void_p), ("hi", ctypes.c_void_p)]
 
 
 class RbsError(RuntimeError):
@@ -73,6 +77,10 @@ def load_library() -> ctypes.CDLL:
                                        vp, f, vp, sz, vp]
     lib.rbs_device_status.restype = i
     lib.rbs_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint), i]
+    lib.rbs_block_stats_box.restype = i
+    lib.rbs_block_stats_box.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsStats, RbsBox, vp]
+    lib.rbs_select_box.restype = i
+    lib.rbs_select_box.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsBox, ctypes.c_double, i, i, i, vp, vp, vp, vp, sz, vp]
     lib.rbs_selftest_device_table.restype = i
     lib.rbs_selftest_device_table.argtypes = []
     lib.rbs_selftest_wait_timeout.restype = i
@@ -249,6 +257,39 @@ def rbs_sparse_prefill(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, mask: 
                                   _ptr(lse), softmax_scale, _ptr(workspace),
                                   0 if workspace is None else workspace.numel(), _stream()), "rbs_sparse_prefill")
     return (out, lse) if return_lse else out
+
+
+def rbs_block_stats_box(K: torch.Tensor, block: int, stats: BlockStats | None = None):
+    """rbs_block_stats plus, from the same read of K, the per-coordinate minima and maxima of every block
+    (App. D.2).  Returns (stats, box_lo [L, Hkv, M, d] fp32, box_hi)."""
+    lib = load_library()
+    if stats is None:
+        stats = alloc_stats(K, block)
+    lo, hi = torch.empty_like(stats.centroid), torch.empty_like(stats.centroid)
+    shape = _shape(None, K, block)
+    _check(lib.rbs_block_stats_box(ctypes.byref(shape), _tensor(K), stats.c_struct(), RbsBox(lo.data_ptr(), hi.data_ptr()),
+                                   _stream()), "rbs_block_stats_box")
+    return stats, lo, hi
+
+
+def rbs_select_box(Q: torch.Tensor, box_lo: torch.Tensor, box_hi: torch.Tensor, block: int, density_param: float = 0.0405,
+                   n_sink: int = 1, n_local: int = 1, n_recent: int = 1, *, debug: bool = False):
+    """The Quest-style comparison selector (Sec. 4.2, Eq. quest_box): box upper bound as the block logit, the same
+    aggregation over the query block, the ceil(density_param (i + 1)) best causal blocks of query block i plus the
+    forced ones.  Returns (mask, density) and, with debug=True, the choice before the union with the forced blocks."""
+    lib = load_library()
+    L, N, Hq, d = Q.shape
+    Hkv = box_lo.shape[1]
+    M = (N + block - 1) // block
+    shape = RbsShape(L, N, Hq, Hkv, d, block)
+    mask = torch.empty(L, Hq, M, (M + 31) // 32, dtype=torch.int32, device=Q.device)
+    density = torch.empty(L, Hq, dtype=torch.float32, device=Q.device)
+    chosen = torch.empty_like(mask) if debug else None
+    ws = torch.empty(max(256, workspace_bytes(RBS_OP_SELECT_BOX, shape)), dtype=torch.uint8, device=Q.device)
+    _check(lib.rbs_select_box(ctypes.byref(shape), _tensor(Q), RbsBox(box_lo.data_ptr(), box_hi.data_ptr()), float(density_param),
+                              n_sink, n_local, n_recent, _ptr(mask), _ptr(density), _ptr(chosen), _ptr(ws), ws.numel(),
+                              _stream()), "rbs_select_box")
+    return (mask, density, chosen) if debug else (mask, density)
 
 
 def prefill_workspace_bytes(L: int, N: int, Hq: int, Hkv: int, block: int, d: int = 128) -> int:

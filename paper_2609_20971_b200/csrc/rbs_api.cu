@@ -68,6 +68,7 @@ extern "C" size_t rbs_workspace_bytes(int op, const rbs_shape* shape) {
   rbs::Dims x = rbs::make_dims(*shape);
   switch (op) {
     case RBS_OP_SELECT: return rbs::select_workspace(x).bytes;
+    case RBS_OP_SELECT_BOX: return rbs::select_box_workspace_bytes(x);
     case RBS_OP_SPARSE_PREFILL:
       return x.B >= 128 ? rbs::prefill_workspace(x.L, x.Hq, x.Hkv, x.M * (x.B / 128), x.G).bytes : 0;
     default: return 0;

@@ -55,6 +55,9 @@ struct PrefillWorkspace {
 };
 PrefillWorkspace prefill_workspace(int L, int Hq, int Hkv, int n_rows, int G);
 
+// Workspace of rbs_select_box (0 for shapes it does not support).
+size_t select_box_workspace_bytes(const Dims& x);
+
 // TMA tensor map over a bf16 [L][N][H][d] tensor with arbitrary (16-byte aligned) strides; box = box_d x box_t.
 rbs_status make_tmap_lthd(::CUtensorMap_st* out, const void* ptr, int L, int N, int H, int d, int64_t sb, int64_t st,
                           int64_t sh, int box_d, int box_t, bool swizzle128);

@@ -16,10 +16,13 @@ namespace rbs {
 // With WPB = 2 (blocks of 256) two neighbouring warps share a block, 128 rows each: they exchange their column
 // sums and their row maxima through shared memory (two bounded mbarrier rendezvous per block), so a block of 256
 // streams like two blocks of 128 instead of needing a 64 KB slot per warp.
-template <int B, int NW, int NS, int WPB>
+// BOX: the same read of K also gives the per-coordinate minima and maxima of each block (the statistics of the
+// Quest-style comparison selector, App. D.2), written to box_lo / box_hi.
+template <int B, int NW, int NS, int WPB, bool BOX>
 __global__ void __launch_bounds__(NW * 32, 1)
 block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, int M, int Hkv, int N,
-                        float* __restrict__ centroid, float* __restrict__ radius, unsigned int* status) {
+                        float* __restrict__ centroid, float* __restrict__ radius, float* __restrict__ box_lo,
+                        float* __restrict__ box_hi, unsigned int* status) {
   constexpr int RW = B / WPB;                 // rows of a block held by one warp
   constexpr uint32_t kPanel = RW * 128;      // bytes of one 64-column panel
   constexpr uint32_t kSlot = 2 * kPanel;
@@ -33,6 +36,7 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
   __shared__ __align__(16) float s_cen[NW][kHeadDim / 2];
   __shared__ __align__(16) float s_sum[WPB == 2 ? NW : 1][kHeadDim];   // a warp's column sums, for its partner
   __shared__ float s_max[WPB == 2 ? NW : 1];
+  __shared__ __align__(16) float s_lo[BOX && WPB == 2 ? NW : 1][kHeadDim], s_hi[BOX && WPB == 2 ? NW : 1][kHeadDim];
   __shared__ __align__(8) uint64_t pair_bar[NG];
 
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -74,7 +78,16 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
     const uint32_t slot = slot0 + buf * kSlot;
     const uint32_t p1_base = slot + (c16 >> 3) * kPanel + (lane & 1) * 8;
     if (!mbar_wait(bar0 + 8 * buf, phase, status, kWaitTmaFull)) break;
+    int idx = t;
+    const int hk = idx % Hkv; idx /= Hkv;
+    const int b = idx % M;
+    const int l = idx / M;
+    // a short last block: TMA filled the rows past the sequence end with zeros; divide by its own size |K_b|
+    const int rows_block = min(B, N - b * B);
+    const int rows_valid = max(0, min(RW, rows_block - part * RW));   // of this warp's rows
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    float lo0 = INFINITY, lo1 = INFINITY, lo2 = INFINITY, lo3 = INFINITY;
+    float hi0 = -INFINITY, hi1 = -INFINITY, hi2 = -INFINITY, hi3 = -INFINITY;
 #pragma unroll 4
     for (int r8 = 0; r8 < RW; r8 += 8) {
 #pragma unroll
@@ -83,27 +96,37 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
         asm volatile("ld.shared.v2.b32 {%0, %1}, [%2];" : "=r"(lo), "=r"(hi)
                      : "r"(p1_base + (r8 + rr) * 128 + ((cp ^ rr) << 4)));
         a0 += bf16lo(lo); a1 += bf16hi(lo); a2 += bf16lo(hi); a3 += bf16hi(hi);
+        if (BOX && r8 + rr < rows_valid) {   // the zero rows past the sequence end are not keys
+          lo0 = fminf(lo0, bf16lo(lo)); lo1 = fminf(lo1, bf16hi(lo)); lo2 = fminf(lo2, bf16lo(hi)); lo3 = fminf(lo3, bf16hi(hi));
+          hi0 = fmaxf(hi0, bf16lo(lo)); hi1 = fmaxf(hi1, bf16hi(lo)); hi2 = fmaxf(hi2, bf16lo(hi)); hi3 = fmaxf(hi3, bf16hi(hi));
+        }
       }
     }
-    int idx = t;
-    const int hk = idx % Hkv; idx /= Hkv;
-    const int b = idx % M;
-    const int l = idx / M;
-    // a short last block: TMA filled the rows past the sequence end with zeros; divide by its own size |K_b|
-    const int rows_block = min(B, N - b * B);
-    const int rows_valid = max(0, min(RW, rows_block - part * RW));   // of this warp's rows
     const float inv_rows = 1.0f / static_cast<float>(rows_block);
     bool pair_ok = true;
     if (WPB == 2) {   // add the partner's column sums (rows past the sequence end arrived as zeros)
       reinterpret_cast<float4*>(s_sum[warp])[lane] = make_float4(a0, a1, a2, a3);
+      if (BOX) {
+        reinterpret_cast<float4*>(s_lo[warp])[lane] = make_float4(lo0, lo1, lo2, lo3);
+        reinterpret_cast<float4*>(s_hi[warp])[lane] = make_float4(hi0, hi1, hi2, hi3);
+      }
       mbar_arrive(smem_u32(&pair_bar[group]));
       pair_ok = mbar_wait(smem_u32(&pair_bar[group]), 0, status, kWaitStageFree);
       const float4 o = reinterpret_cast<const float4*>(s_sum[warp ^ 1])[lane];
       a0 += o.x; a1 += o.y; a2 += o.z; a3 += o.w;
+      if (BOX) {
+        const float4 ol = reinterpret_cast<const float4*>(s_lo[warp ^ 1])[lane], oh = reinterpret_cast<const float4*>(s_hi[warp ^ 1])[lane];
+        lo0 = fminf(lo0, ol.x); lo1 = fminf(lo1, ol.y); lo2 = fminf(lo2, ol.z); lo3 = fminf(lo3, ol.w);
+        hi0 = fmaxf(hi0, oh.x); hi1 = fmaxf(hi1, oh.y); hi2 = fmaxf(hi2, oh.z); hi3 = fmaxf(hi3, oh.w);
+      }
     }
     const float4 cen = make_float4(a0 * inv_rows, a1 * inv_rows, a2 * inv_rows, a3 * inv_rows);
     const int64_t blk = (static_cast<int64_t>(l) * Hkv + hk) * M + b;
     if (part == 0) reinterpret_cast<float4*>(centroid + blk * kHeadDim)[lane] = cen;
+    if (BOX && part == 0) {
+      reinterpret_cast<float4*>(box_lo + blk * kHeadDim)[lane] = make_float4(lo0, lo1, lo2, lo3);
+      reinterpret_cast<float4*>(box_hi + blk * kHeadDim)[lane] = make_float4(hi0, hi1, hi2, hi3);
+    }
 
     float q[RJ];
 #pragma unroll
@@ -160,8 +183,9 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
   }
 }
 
-template <int B, int NW, int NS, int WPB>
-static rbs_status launch_stats_warp(const rbs_tensor& K, const Dims& x, const rbs_stats& stats, cudaStream_t s) {
+template <int B, int NW, int NS, int WPB, bool BOX>
+static rbs_status launch_stats_warp(const rbs_tensor& K, const Dims& x, const rbs_stats& stats, float* box_lo, float* box_hi,
+                                    cudaStream_t s) {
   CUtensorMap tm;
   rbs_status st = make_tmap_lthd(&tm, K.ptr, x.L, x.N, x.Hkv, x.d, K.stride_batch, K.stride_token, K.stride_head,
                                  64, B / WPB, true);
@@ -169,19 +193,21 @@ static rbs_status launch_stats_warp(const rbs_tensor& K, const Dims& x, const rb
   unsigned int* status = device_status_ptr();
   if (status == nullptr) return RBS_ERR_CUDA;
   const size_t smem = static_cast<size_t>(NW) * NS * (B / WPB) * 256;
-  auto kern = block_stats_warp_kernel<B, NW, NS, WPB>;
+  auto kern = block_stats_warp_kernel<B, NW, NS, WPB, BOX>;
   if ((st = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem)) != RBS_OK) return st;
   const long long n_tiles = static_cast<long long>(x.L) * x.Hkv * x.M;
   long long want = (n_tiles + NW / WPB - 1) / (NW / WPB);
   const int grid = static_cast<int>(want < sm_count() ? want : sm_count());
-  kern<<<grid, NW * 32, smem, s>>>(tm, static_cast<int>(n_tiles), x.M, x.Hkv, x.N, stats.centroid, stats.radius, status);
+  kern<<<grid, NW * 32, smem, s>>>(tm, static_cast<int>(n_tiles), x.M, x.Hkv, x.N, stats.centroid, stats.radius, box_lo,
+                                   box_hi, status);
   RBS_CUDA_OK(cudaGetLastError());
   return RBS_OK;
 }
 
 }  // namespace rbs
 
-extern "C" rbs_status rbs_block_stats(const rbs_shape* shape, rbs_tensor K, rbs_stats stats, void* stream) {
+static rbs_status block_stats_impl(const rbs_shape* shape, rbs_tensor K, rbs_stats stats, float* box_lo, float* box_hi,
+                                   void* stream) {
   using namespace rbs;
   rbs_status st = check_shape(shape);
   if (st != RBS_OK) return st;
@@ -189,6 +215,9 @@ extern "C" rbs_status rbs_block_stats(const rbs_shape* shape, rbs_tensor K, rbs_
   if (st != RBS_OK) return st;
   if (stats.centroid == nullptr || stats.radius == nullptr) return RBS_ERR_INVALID_ARG;
   if (reinterpret_cast<uintptr_t>(stats.centroid) % 16 != 0) return RBS_ERR_INVALID_ARG;
+  const bool box = box_lo != nullptr;
+  if (box && (box_hi == nullptr || reinterpret_cast<uintptr_t>(box_lo) % 16 != 0 || reinterpret_cast<uintptr_t>(box_hi) % 16 != 0))
+    return RBS_ERR_INVALID_ARG;
   Dims x = make_dims(*shape);
   const long long n_tiles = static_cast<long long>(x.L) * x.Hkv * x.M;
   if (n_tiles > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
@@ -198,7 +227,21 @@ extern "C" rbs_status rbs_block_stats(const rbs_shape* shape, rbs_tensor K, rbs_
   //            32.4 us; three warps with two 32 KB slots each: 46 us, compute-bound)
   //   B = 64:  seven warps with two 16 KB slots each used in turn      28.7 us   (fourteen single-slot warps: 31.1 us)
   //   B = 256: six warps in pairs, 128 rows and a 32 KB slot each      35.7 us   (three warps, 64 KB slots: 58 us)
-  if (x.B == 256) return launch_stats_warp<256, 6, 1, 2>(K, x, stats, s);
-  if (x.B == 128) return launch_stats_warp<128, 12, 1, 2>(K, x, stats, s);
-  return launch_stats_warp<64, 7, 2, 1>(K, x, stats, s);
+  if (box) {
+    if (x.B == 256) return launch_stats_warp<256, 6, 1, 2, true>(K, x, stats, box_lo, box_hi, s);
+    if (x.B == 128) return launch_stats_warp<128, 12, 1, 2, true>(K, x, stats, box_lo, box_hi, s);
+    return launch_stats_warp<64, 7, 2, 1, true>(K, x, stats, box_lo, box_hi, s);
+  }
+  if (x.B == 256) return launch_stats_warp<256, 6, 1, 2, false>(K, x, stats, nullptr, nullptr, s);
+  if (x.B == 128) return launch_stats_warp<128, 12, 1, 2, false>(K, x, stats, nullptr, nullptr, s);
+  return launch_stats_warp<64, 7, 2, 1, false>(K, x, stats, nullptr, nullptr, s);
+}
+
+extern "C" rbs_status rbs_block_stats(const rbs_shape* shape, rbs_tensor K, rbs_stats stats, void* stream) {
+  return block_stats_impl(shape, K, stats, nullptr, nullptr, stream);
+}
+
+extern "C" rbs_status rbs_block_stats_box(const rbs_shape* shape, rbs_tensor K, rbs_stats stats, rbs_box box, void* stream) {
+  if (box.lo == nullptr || box.hi == nullptr) return RBS_ERR_INVALID_ARG;
+  return block_stats_impl(shape, K, stats, box.lo, box.hi, stream);
 }

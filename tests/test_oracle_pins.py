@@ -462,3 +462,70 @@ def test_group_union_is_a_superset_with_additive_density_bound():
     rho = [orc.density(f) for f in heads]
     assert max(rho) <= orc.density(u) <= sum(rho)
     assert np.array_equal(orc.group_union([heads[0]]), heads[0])
+
+
+# ----------------------------------------------------------------------------- Sec. 4.2 / App. D.2: Quest-style box selector
+def test_box_stats_and_bound_against_the_worked_examples_and_brute_force():
+    ex = GOLDEN["cross_polytope"]
+    keys, q = np.array(ex["keys"], float), np.array(ex["q"], float)
+    lo, hi = orc.box_stats(keys, 4)
+    assert np.array_equal(lo[0], [-1, -1]) and np.array_equal(hi[0], [1, 1])
+    assert orc.box_logits(q[None, :], lo, hi)[0, 0] == pytest.approx(ex["U_box"])
+    ex = GOLDEN["thin_box"]
+    e = ex["eps"]
+    keys = np.array([[1, 0], [-1, 0], [0, e], [0, -e]], float)
+    lo, hi = orc.box_stats(keys, 4)
+    assert orc.box_logits(np.array([ex["q"]], float), lo, hi)[0, 0] == pytest.approx(e * ex["U_box_over_eps"])
+    # random blocks: per-coordinate extrema by pure Python; the bound dominates every token logit and equals
+    # q.v + |q|.h with the box centre v and half-width h (App. D.2)
+    g = rng(20)
+    B, d, M = 6, 5, 4
+    K = g.normal(size=(B * M, d)) * g.uniform(0.2, 2.0, size=(B * M, 1))
+    Q = g.normal(size=(7, d))
+    lo, hi = orc.box_stats(K, B)
+    for b in range(M):
+        rows = [list(map(float, K[b * B + t])) for t in range(B)]
+        assert np.array_equal(lo[b], [min(r[j] for r in rows) for j in range(d)])
+        assert np.array_equal(hi[b], [max(r[j] for r in rows) for j in range(d)])
+    U = orc.box_logits(Q, lo, hi)
+    token_max = np.stack([(Q @ K[b * B:(b + 1) * B].T).max(axis=1) for b in range(M)], axis=1)
+    assert np.all(U >= token_max - 1e-12)
+    v, h = (hi + lo) / 2, (hi - lo) / 2
+    assert np.allclose(U, Q @ v.T + np.abs(Q) @ h.T, rtol=1e-13, atol=1e-13)
+    # a short last block uses its own keys only
+    lo2, hi2 = orc.box_stats(K[:B * M - 2], B)
+    assert np.array_equal(lo2[-1], K[B * (M - 1):B * M - 2].min(0)) and np.array_equal(lo2[:-1], lo[:-1])
+
+
+def test_top_fraction_counts_ties_and_extremes():
+    S = np.array([5.0, 1.0, 3.0, 3.0, 2.0, 0.5, 4.0, 0.1])
+    assert orc.top_fraction(S, 0.25).sum() == 2 and orc.top_fraction(S, 0.25)[[0, 6]].all()
+    assert orc.top_fraction(S, 0.26).sum() == 4          # ceil(2.08) = 3, and the tie with the third score is kept
+    assert orc.top_fraction(S, 1.0).all() and orc.top_fraction(S, 1e-9).sum() == 1
+    assert orc.top_fraction(np.array([2.0]), 0.0405).all()
+
+
+def test_box_selection_closed_form_scene_and_invariants():
+    # identical queries sqrt(d) e1; block b holds keys x_b e1 +/- w_b e2: box logit / sqrt(d) = x_b exactly
+    # (the queries have no e2 component), so row i keeps the ceil(delta (i + 1)) largest x_b, b <= i
+    B, d = 4, 16
+    x = np.array([0.0, -1.0, 2.0, 0.5, -0.2, 3.0, 0.4, -1.4, 1.0, 0.9])
+    Q, K = _scene(x, np.linspace(0.1, 2.0, len(x)), d, B)
+    lo, hi = orc.box_stats(K, B)
+    M = len(x)
+    sel = orc.select_head_box(Q, lo, hi, B, 0.3, 0, 0, 0)
+    for i in range(M):
+        k = int(math.ceil(0.3 * (i + 1)))
+        want = np.zeros(i + 1, bool)
+        want[np.argsort(-x[:i + 1], kind="stable")[:k]] = True
+        assert np.array_equal(sel.final[i, :i + 1], want) and not sel.final[i, i + 1:].any()
+        kth = np.sort(x[:i + 1])[::-1][k - 1]
+        assert np.allclose(sel.margin[i, :i + 1], np.abs(np.exp(x[:i + 1] - kth) - 1.0), rtol=1e-12, atol=1e-14)
+    assert sel.density == pytest.approx(sum(int(math.ceil(0.3 * (i + 1))) for i in range(M)) / (M * (M + 1) / 2))
+    # forced blocks are united in; a larger density parameter never removes a block
+    Qr, Kr, _ = _random_head(21, M=20, B=8)
+    lo, hi = orc.box_stats(Kr, 8)
+    a = orc.select_head_box(Qr, lo, hi, 8, 0.1, 1, 1, 1)
+    b2 = orc.select_head_box(Qr, lo, hi, 8, 0.25, 1, 1, 1)
+    assert np.array_equal(a.final, a.chosen | a.forced) and np.all(b2.final | ~a.final) and b2.density >= a.density
+    assert a.final[-1, :].all() and a.final[:, 0].all() and np.diag(a.final).all()
