@@ -254,6 +254,19 @@ RBS_API rbs_status rbs_mask_group_union(const rbs_shape* shape, int q_start_bloc
                                         float* density, void* stream);
 
 /*
+ * rbs_sparse_prefill for group-shared masks: the caller states that the G query heads of every KV group have identical
+ * mask rows (as rbs_mask_group_union leaves them).  Two heads of a group are then served by one thread block that brings
+ * every selected K/V tile into shared memory once for both (head-packed query tiles), instead of once per head.  The
+ * paper's selector is per query head (Sec. 3.2), so this execution variant has no counterpart there; the attention it
+ * computes is Sec. 3.3's.  Arguments and outputs as rbs_sparse_prefill (whole sequence only, no workspace); the mask is
+ * read from the first head of each pair.  Needs block >= 128 and an even group size (RBS_ERR_UNSUPPORTED otherwise)
+ * and a mask (RBS_ERR_INVALID_ARG for NULL).
+ */
+RBS_API rbs_status rbs_sparse_prefill_grouped(const rbs_shape* shape, rbs_tensor Q, rbs_tensor K, rbs_tensor V,
+                                              const uint32_t* mask, rbs_tensor O, float* lse, float softmax_scale,
+                                              void* stream);
+
+/*
  * Kernels that wait on hardware barriers (TMA arrival, tensor-core completion) give every wait an
  * iteration limit.  A wait that runs out records a non-zero code in a device-side status word, lets the
  * kernel drain and return, and leaves the CUDA context usable; outputs of that launch are then

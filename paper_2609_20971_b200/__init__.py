@@ -5,7 +5,7 @@ The Python names mirror the C entry points.  Importing this package does not loa
 the first call does, and raises if it has not been built.
 """
 from .binding import (BlockStats, RbsError, alloc_stats, load_library, rbs_block_stats, rbs_block_stats_box, rbs_device_status, rbs_select_box,
-                      rbs_mask_group_union, rbs_select, rbs_select_chunk, rbs_select_static, rbs_sparse_prefill_chunk, rbs_sparse_prefill, workspace_bytes)
+                      rbs_mask_group_union, rbs_select, rbs_select_chunk, rbs_select_static, rbs_sparse_prefill_chunk, rbs_sparse_prefill, rbs_sparse_prefill_grouped, workspace_bytes)
 
 __all__ = ["BlockStats", "RbsError", "alloc_stats", "load_library", "rbs_block_stats", "rbs_block_stats_box", "rbs_device_status", "rbs_select_box",
-           "rbs_mask_group_union", "rbs_select", "rbs_select_chunk", "rbs_select_static", "rbs_sparse_prefill_chunk", "rbs_sparse_prefill", "workspace_bytes"]
+           "rbs_mask_group_union", "rbs_select", "rbs_select_chunk", "rbs_select_static", "rbs_sparse_prefill_chunk", "rbs_sparse_prefill", "rbs_sparse_prefill_grouped", "workspace_bytes"]

@@ -75,6 +75,8 @@ def load_library() -> ctypes.CDLL:
     lib.rbs_sparse_prefill.restype = i
     lib.rbs_sparse_prefill.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsTensor, RbsTensor, vp, RbsTensor,
                                        vp, f, vp, sz, vp]
+    lib.rbs_sparse_prefill_grouped.restype = i
+    lib.rbs_sparse_prefill_grouped.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsTensor, RbsTensor, vp, RbsTensor, vp, f, vp]
     lib.rbs_device_status.restype = i
     lib.rbs_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint), i]
     lib.rbs_block_stats_box.restype = i
@@ -290,6 +292,21 @@ def rbs_select_box(Q: torch.Tensor, box_lo: torch.Tensor, box_hi: torch.Tensor, 
                               n_sink, n_local, n_recent, _ptr(mask), _ptr(density), _ptr(chosen), _ptr(ws), ws.numel(),
                               _stream()), "rbs_select_box")
     return (mask, density, chosen) if debug else (mask, density)
+
+
+def rbs_sparse_prefill_grouped(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, mask: torch.Tensor, block: int, *,
+                               out: torch.Tensor | None = None, return_lse: bool = False, softmax_scale: float = 0.0):
+    """rbs_sparse_prefill for masks that are identical inside every KV group (after rbs_mask_group_union): two heads
+    of a group share one stream of K/V tiles."""
+    lib = load_library()
+    L, N, Hq, d = Q.shape
+    shape = RbsShape(L, N, Hq, K.shape[2], d, block)
+    if out is None:
+        out = torch.empty_like(Q)
+    lse = torch.empty(L, Hq, N, dtype=torch.float32, device=Q.device) if return_lse else None
+    _check(lib.rbs_sparse_prefill_grouped(ctypes.byref(shape), _tensor(Q), _tensor(K), _tensor(V), _ptr(mask), _tensor(out),
+                                          _ptr(lse), softmax_scale, _stream()), "rbs_sparse_prefill_grouped")
+    return (out, lse) if return_lse else out
 
 
 def prefill_workspace_bytes(L: int, N: int, Hq: int, Hkv: int, block: int, d: int = 128) -> int:

@@ -6,65 +6,9 @@
 // block of 64.
 #include "rbs_common.cuh"
 #include "rbs_sm100.cuh"
+#include "rbs_prefill.cuh"
 
 namespace rbs {
-
-struct PrefillParams {
-  const __nv_bfloat16* Q; int64_t qsb, qst, qsh;
-  const __nv_bfloat16* K; int64_t ksb, kst, ksh;
-  const __nv_bfloat16* V; int64_t vsb, vst, vsh;
-  __nv_bfloat16* O; int64_t osb, ost, osh;
-  const uint32_t* mask;  // nullptr: dense
-  float* lse;            // nullable
-  int M, W, L, Hq, G, N;
-  int R;   // 128-row tiles per block (tensor-core path): block / 128
-  int q0, Mq, Nq;   // this call's queries: first query block (global index), number of blocks, number of tokens
-  int band_rows;    // 128-row query tiles per band of the tile order (tensor-core path)
-  float scale_log2;
-  // Row-length-aware schedule (null: tiles in their static order, one CTA per tile).  One int4 per CTA:
-  // x = position of the tile in its group's static order (-1: nothing to do), [y, z) = range of 128-key sub-blocks
-  // this item attends, w = slot of its partial result (-1: the item is a whole row and writes O itself).
-  const int4* items;
-  int items_per_group;
-  float* part_o;    // [slot][128 rows][128] unnormalised O of a part, fp32
-  float* part_ml;   // [slot][2][128]        running maximum (log2 units) and row sum of a part
-};
-
-// Rows longer than this many 128-key sub-blocks are cut into parts of equal length that run as separate CTAs and are
-// merged afterwards; the cut depends only on the row itself, so a row is treated the same in every call.
-constexpr int kSplitCap = 256;
-constexpr int kSplitMaxParts = 4;      // parts per split row
-constexpr int kSplitRowsPerGroup = 8;  // split rows per (band, batch, KV head) group: its longest ones
-constexpr int kSplitSlotsPerGroup = kSplitRowsPerGroup * kSplitMaxParts;
-constexpr int kExtraItemsPerGroup = kSplitRowsPerGroup * (kSplitMaxParts - 1);
-
-// next selected key block after `cur` (cur = -1 to start), restricted to b <= i; -1 when exhausted
-__device__ __forceinline__ int next_block(const uint32_t* __restrict__ row, int cur, int i) {
-  int b = cur + 1;
-  if (row == nullptr) return b <= i ? b : -1;
-  while (b <= i) {
-    uint32_t w = __ldg(row + (b >> 5)) >> (b & 31);
-    if (w) {
-      b += __ffs(w) - 1;
-      return b <= i ? b : -1;
-    }
-    b = (b | 31) + 1;
-  }
-  return -1;
-}
-
-// Tensor-core path, blocks of R x 128 tokens: the kernel works on 128-row query tiles T and 128-key sub-blocks kb.
-// Sub-block kb belongs to mask block kb / R; tile T (of query block T / R) attends sub-blocks kb <= T of the selected
-// blocks, kb == T being the diagonal one.  Returns the next sub-block after `cur` (-1 to start), or -1.
-__device__ __forceinline__ int next_kb(const uint32_t* __restrict__ row, int cur, int i, int R, int T) {
-  int kb = cur + 1;
-  if (kb > T) return -1;
-  const int b = kb / R;
-  const int nb = next_block(row, b - 1, i);   // first selected block >= b
-  if (nb < 0) return -1;
-  if (nb != b) kb = nb * R;
-  return kb <= T ? kb : -1;
-}
 
 template <int B>
 __global__ void __launch_bounds__(B * 2, 1)
@@ -263,8 +207,6 @@ prefill_mma_kernel(const PrefillParams p) {
 // against its exact maximum only when its sum reaches kSumLimit, so P stays below kSumLimit and O is rescaled rarely.
 // ---------------------------------------------------------------------------------------------
 constexpr int kPfThreads = 256;
-// A half-row of P whose sum reaches this value makes the row adopt the half's exact maximum.
-constexpr float kSumLimit = 16384.0f;
 // Of every (kPolyEvery + 1) groups of four logits, one pair is exponentiated by polynomial on the FMA pipe instead of
 // by ex2 (0: every group = 50 % of the exps, 1: 25 %, 3: 12.5 %, 16: none).  The polynomial relieves the exp unit but
 // costs about six instructions per element, and the launch is bound by power, not by the exp unit: on the 128K
@@ -1200,9 +1142,10 @@ static rbs_status launch_prefill(const PrefillParams& p, cudaStream_t s) {
 
 }  // namespace rbs
 
+// grouped: the caller states that the query heads of a KV group have identical mask rows (rbs_sparse_prefill_grouped)
 static rbs_status prefill_impl(const rbs_shape* shape, int q_start_block, int n_q_tokens, rbs_tensor Q, rbs_tensor K,
                                rbs_tensor V, const uint32_t* mask, rbs_tensor O, float* lse, float softmax_scale,
-                               void* workspace, size_t workspace_bytes, void* stream) {
+                               void* workspace, size_t workspace_bytes, void* stream, bool grouped = false) {
   using namespace rbs;
   rbs_status st = check_shape(shape);
   if (st != RBS_OK) return st;
@@ -1225,6 +1168,12 @@ static rbs_status prefill_impl(const rbs_shape* shape, int q_start_block, int n_
   p.scale_log2 = scale * kLog2e;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   p.R = x.B / 128;
+  p.band_rows = 0; p.items = nullptr; p.items_per_group = 0; p.part_o = nullptr; p.part_ml = nullptr;
+  if (grouped) {
+    if (mask == nullptr) return RBS_ERR_INVALID_ARG;
+    if (x.B < 128 || x.G % 2 != 0) return RBS_ERR_UNSUPPORTED;
+    return launch_prefill_pair(p, Q, K, V, x.Hkv, 0, s);
+  }
   if (x.B >= 128 && mask != nullptr && workspace != nullptr) {   // checked before anything touches the GPU
     const PrefillWorkspace w = prefill_workspace(x.L, x.Hq, x.Hkv, x.M * p.R, x.G);
     if (workspace_bytes < w.bytes || reinterpret_cast<uintptr_t>(workspace) % 256 != 0) return RBS_ERR_WORKSPACE;
@@ -1257,4 +1206,10 @@ extern "C" rbs_status rbs_sparse_prefill_chunk(const rbs_shape* shape, int q_sta
   if (n_q_tokens <= 0) return RBS_ERR_INVALID_ARG;
   return prefill_impl(shape, q_start_block, n_q_tokens, Q, K, V, mask, O, lse, softmax_scale, workspace,
                       workspace_bytes, stream);
+}
+
+extern "C" rbs_status rbs_sparse_prefill_grouped(const rbs_shape* shape, rbs_tensor Q, rbs_tensor K, rbs_tensor V,
+                                                 const uint32_t* mask, rbs_tensor O, float* lse, float softmax_scale,
+                                                 void* stream) {
+  return prefill_impl(shape, -1, -1, Q, K, V, mask, O, lse, softmax_scale, nullptr, 0, stream, true);
 }

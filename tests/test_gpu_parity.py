@@ -534,3 +534,36 @@ def test_long_rows_are_split_and_merged(B, M, tail):
     oc, lc = rbs_sparse_prefill_chunk(Qg[:, q0 * B:], Kg, Vg, mask[:, :, q0:].contiguous(), B, q0, return_lse=True,
                                       workspace=ws)
     assert torch.equal(oc, O[:, q0 * B:]) and torch.equal(lc, lse[:, :, q0 * B:])
+
+
+def test_grouped_attention_under_group_shared_masks():
+    """Head-packed query tiles: with the masks of a KV group made identical (rbs_mask_group_union) two heads of the group
+    share one stream of K/V tiles.  Against the oracle (attention over the oracle's union of the GPU's per-head masks) and
+    against the one-head-per-CTA kernel on the same mask."""
+    from paper_2609_20971_b200 import rbs_sparse_prefill_grouped
+    for cfg in (SynthConfig("grouped", L=2, N=128 * 45 + 50, Hq=8, Hkv=2, B=128, sigma=(0.1, 1.0), seed=62),
+                SynthConfig("grouped256", N=256 * 21, Hq=4, Hkv=2, B=256, sigma=0.6, seed=63)):
+        Q, K, V = make_inputs(cfg)
+        dev = torch.device("cuda:0")
+        Qg, Kg, Vg = Q.to(dev), K.to(dev), V.to(dev)
+        stats = rbs_block_stats(Kg, cfg.B)
+        mask, dens = rbs_select(Qg, stats, cfg.B, cfg.alpha_base, cfg.alpha_rescue, 1, 1, 1)
+        per_head = unpack_mask(mask, cfg.M)
+        rbs_mask_group_union(mask, dens, cfg.Hkv, cfg.B, cfg.N)
+        O, lse = rbs_sparse_prefill_grouped(Qg, Kg, Vg, mask, cfg.B, return_lse=True)
+        O1, lse1 = rbs_sparse_prefill(Qg, Kg, Vg, mask, cfg.B, return_lse=True)
+        torch.cuda.synchronize()
+        assert (O.float() - O1.float()).abs().max().item() <= OUT_MAX_ABS
+        assert torch.allclose(lse, lse1, atol=2e-3, rtol=1e-4)
+        M, B, G = cfg.M, cfg.B, cfg.Hq // cfg.Hkv
+        Q64, K64, V64 = to_f64(Q), to_f64(K), to_f64(V)
+        Onp, lnp = O.float().cpu().numpy(), lse.cpu().numpy()
+        for l in range(cfg.L):
+            for h in (0, 3, cfg.Hq - 1):
+                hk = h // G
+                want_mask = orc.group_union([per_head[l, hk * G + g] for g in range(G)])
+                for i in (0, 1, M // 2, M - 1):
+                    ref, lref = orc.masked_attention_block(Q64[l, :, h], K64[l, :, hk], V64[l, :, hk], want_mask[i], i, B)
+                    t0, t1 = i * B, min(cfg.N, (i + 1) * B)
+                    _check_output(Onp[l, t0:t1, h], ref)
+                    assert np.allclose(lnp[l, h, t0:t1], lref, atol=2e-3, rtol=1e-4)
