@@ -267,6 +267,26 @@ RBS_API rbs_status rbs_sparse_prefill_grouped(const rbs_shape* shape, rbs_tensor
                                               void* stream);
 
 /*
+ * A batch of prompts of different lengths packed back to back along the token axis (no padding).  Every prompt is
+ * selected and attended on its own, exactly as by rbs_block_stats + rbs_select + rbs_sparse_prefill on its rows
+ * (Sec. 4.1: requests are not concatenated into one causal sequence); results are bit-identical to those calls.
+ *   cu_seqlens   HOST array of n_prompts + 1 ints: cu_seqlens[0] = 0, prompt k holds tokens [cu_seqlens[k], cu_seqlens[k+1])
+ *   Q, O         packed [T][Hq][d]; K, V packed [T][Hkv][d] (stride_token, stride_head in elements; stride_batch ignored)
+ *   density      device, [n_prompts][Hq] fp32
+ *   workspace    device, rbs_varlen_workspace_bytes(...) bytes, 256-byte aligned: statistics, mask and selector scratch
+ *                of the longest prompt, reused from prompt to prompt in stream order (nothing is allocated, no tensor
+ *                outlives the call; the per-prompt masks and statistics are not returned).
+ * Errors: RBS_ERR_INVALID_ARG for a malformed cu_seqlens (not starting at 0, not strictly increasing), otherwise as the
+ * three calls.  All prompts are enqueued on `stream` one after the other.
+ */
+RBS_API size_t rbs_varlen_workspace_bytes(int n_prompts, const int* cu_seqlens, int n_q_heads, int n_kv_heads,
+                                          int head_dim, int block);
+RBS_API rbs_status rbs_prefill_varlen(int n_prompts, const int* cu_seqlens, int n_q_heads, int n_kv_heads, int head_dim,
+                                      int block, rbs_tensor Q, rbs_tensor K, rbs_tensor V, rbs_tensor O, float alpha_base,
+                                      float alpha_rescue, int n_sink, int n_local, int n_recent, float* density,
+                                      void* workspace, size_t workspace_bytes, void* stream);
+
+/*
  * Kernels that wait on hardware barriers (TMA arrival, tensor-core completion) give every wait an
  * iteration limit.  A wait that runs out records a non-zero code in a device-side status word, lets the
  * kernel drain and return, and leaves the CUDA context usable; outputs of that launch are then

@@ -77,6 +77,11 @@ def load_library() -> ctypes.CDLL:
                                        vp, f, vp, sz, vp]
     lib.rbs_sparse_prefill_grouped.restype = i
     lib.rbs_sparse_prefill_grouped.argtypes = [ctypes.POINTER(RbsShape), RbsTensor, RbsTensor, RbsTensor, vp, RbsTensor, vp, f, vp]
+    lib.rbs_varlen_workspace_bytes.restype = sz
+    lib.rbs_varlen_workspace_bytes.argtypes = [i, ctypes.POINTER(ctypes.c_int), i, i, i, i]
+    lib.rbs_prefill_varlen.restype = i
+    lib.rbs_prefill_varlen.argtypes = [i, ctypes.POINTER(ctypes.c_int), i, i, i, i, RbsTensor, RbsTensor, RbsTensor, RbsTensor,
+                                       f, f, i, i, i, vp, vp, sz, vp]
     lib.rbs_device_status.restype = i
     lib.rbs_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint), i]
     lib.rbs_block_stats_box.restype = i
@@ -307,6 +312,39 @@ def rbs_sparse_prefill_grouped(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor
     _check(lib.rbs_sparse_prefill_grouped(ctypes.byref(shape), _tensor(Q), _tensor(K), _tensor(V), _ptr(mask), _tensor(out),
                                           _ptr(lse), softmax_scale, _stream()), "rbs_sparse_prefill_grouped")
     return (out, lse) if return_lse else out
+
+
+def rbs_prefill_varlen(Q: torch.Tensor, K: torch.Tensor, V: torch.Tensor, cu_seqlens, block: int, *, out=None,
+                       alpha_base: float = 0.22, alpha_rescue: float = 0.18, n_sink: int = 1, n_local: int = 1,
+                       n_recent: int = 1, workspace: torch.Tensor | None = None):
+    """Prompts of different lengths packed along the token axis: Q [T, Hq, d], K, V [T, Hkv, d]; `cu_seqlens` host
+    ints (n + 1).  One library call for the whole batch, one reusable workspace.  Returns (O [T, Hq, d],
+    density [n, Hq])."""
+    lib = load_library()
+    cu = [int(c) for c in cu_seqlens]
+    n = len(cu) - 1
+    arr = (ctypes.c_int * len(cu))(*cu)
+    T, Hq, d = Q.shape
+    Hkv = K.shape[1]
+    if out is None:
+        out = torch.empty_like(Q)
+    need = int(lib.rbs_varlen_workspace_bytes(n, arr, Hq, Hkv, d, block))
+    if need == 0:
+        raise RbsError("rbs_prefill_varlen: cu_seqlens must start at 0 and increase strictly, and the shape must be supported")
+    if cu[-1] != T:
+        raise RbsError("rbs_prefill_varlen: cu_seqlens must end at the number of packed tokens")
+    if workspace is None:
+        workspace = torch.empty(need, dtype=torch.uint8, device=Q.device)
+    density = torch.empty(n, Hq, dtype=torch.float32, device=Q.device)
+
+    def packed(t):
+        if t.dim() != 3 or t.dtype != torch.bfloat16 or not t.is_cuda or t.stride(2) != 1:
+            raise RbsError("expected CUDA bf16 tensors [tokens, heads, head_dim] with head_dim contiguous")
+        return RbsTensor(t.data_ptr(), 0, t.stride(0), t.stride(1))
+    _check(lib.rbs_prefill_varlen(n, arr, Hq, Hkv, d, block, packed(Q), packed(K), packed(V), packed(out), alpha_base,
+                                  alpha_rescue, n_sink, n_local, n_recent, _ptr(density), _ptr(workspace), workspace.numel(),
+                                  _stream()), "rbs_prefill_varlen")
+    return out, density
 
 
 def prefill_workspace_bytes(L: int, N: int, Hq: int, Hkv: int, block: int, d: int = 128) -> int:

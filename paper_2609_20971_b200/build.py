@@ -9,7 +9,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "librbs_b200.so")
-SOURCES = ["rbs_api.cu", "rbs_tmap.cu", "rbs_stats.cu", "rbs_select.cu", "rbs_prefill.cu", "rbs_prefill_pair.cu", "rbs_union.cu", "rbs_box.cu"]
+SOURCES = ["rbs_api.cu", "rbs_tmap.cu", "rbs_stats.cu", "rbs_select.cu", "rbs_prefill.cu", "rbs_prefill_pair.cu", "rbs_union.cu", "rbs_box.cu", "rbs_varlen.cu"]
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
     "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden",

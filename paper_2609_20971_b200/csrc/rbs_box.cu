@@ -286,6 +286,7 @@ extern "C" rbs_status rbs_select_box(const rbs_shape* shape, rbs_tensor Q, rbs_b
                                      int n_local, int n_recent, uint32_t* mask, float* density, uint32_t* dbg_chosen_mask,
                                      void* workspace, size_t workspace_bytes, void* stream) {
   using namespace rbs;
+  rbs::NvtxRange nvtx_range("rbs_select_box");
   rbs_status st = check_shape(shape);
   if (st != RBS_OK) return st;
   if ((st = check_tensor(Q)) != RBS_OK) return st;

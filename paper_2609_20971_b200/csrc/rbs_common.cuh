@@ -7,6 +7,8 @@
 
 #include <mutex>
 
+#include <nvtx3/nvToolsExt.h>
+
 #include "rbs.h"
 
 struct CUtensorMap_st;
@@ -94,6 +96,14 @@ class PerDevice {
   std::mutex lock_;
   bool have_[kMaxDevices] = {};
   T value_[kMaxDevices] = {};
+};
+
+// Named range around an entry point's host work, visible in NVIDIA's timeline tools (a no-op when none is attached).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+  NvtxRange(const NvtxRange&) = delete;
+  NvtxRange& operator=(const NvtxRange&) = delete;
 };
 
 #define RBS_CUDA_OK(expr)                               \

@@ -1147,6 +1147,7 @@ static rbs_status prefill_impl(const rbs_shape* shape, int q_start_block, int n_
                                rbs_tensor V, const uint32_t* mask, rbs_tensor O, float* lse, float softmax_scale,
                                void* workspace, size_t workspace_bytes, void* stream, bool grouped = false) {
   using namespace rbs;
+  rbs::NvtxRange nvtx_range("rbs_sparse_prefill");
   rbs_status st = check_shape(shape);
   if (st != RBS_OK) return st;
   if ((st = check_tensor(Q)) != RBS_OK || (st = check_tensor(K)) != RBS_OK || (st = check_tensor(V)) != RBS_OK ||

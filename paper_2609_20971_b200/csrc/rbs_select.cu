@@ -664,6 +664,7 @@ static rbs_status select_impl(const rbs_shape* shape, int q_start_block, int n_q
                               float* density, uint32_t* dbg_base_mask, uint32_t* dbg_rescue_mask,
                               void* workspace, size_t workspace_bytes, void* stream) {
   using namespace rbs;
+  rbs::NvtxRange nvtx_range("rbs_select");
   rbs_status st = check_shape(shape);
   if (st != RBS_OK) return st;
   st = check_tensor(Q);

@@ -209,6 +209,7 @@ static rbs_status launch_stats_warp(const rbs_tensor& K, const Dims& x, const rb
 static rbs_status block_stats_impl(const rbs_shape* shape, rbs_tensor K, rbs_stats stats, float* box_lo, float* box_hi,
                                    void* stream) {
   using namespace rbs;
+  rbs::NvtxRange nvtx_range("rbs_block_stats");
   rbs_status st = check_shape(shape);
   if (st != RBS_OK) return st;
   st = check_tensor(K);

@@ -151,3 +151,18 @@ def test_wait_timeout_selftest_argument_checks(lib):
     assert lib.rbs_selftest_wait_timeout(0, p, None) == INVALID
     assert lib.rbs_selftest_wait_timeout(1 << 20, p, None) == INVALID      # only short limits are accepted
     assert lib.rbs_selftest_wait_timeout(1024, None, None) == INVALID
+
+
+def test_varlen_argument_checks(lib):
+    lib.rbs_varlen_workspace_bytes.restype = ctypes.c_size_t
+    good = (ctypes.c_int * 4)(0, 300, 1000, 1001)
+    need = lib.rbs_varlen_workspace_bytes(3, good, 4, 2, 128, 128)
+    assert need > 0 and need % 256 == 0
+    assert lib.rbs_varlen_workspace_bytes(3, (ctypes.c_int * 4)(1, 300, 1000, 1001), 4, 2, 128, 128) == 0     # not from 0
+    assert lib.rbs_varlen_workspace_bytes(3, (ctypes.c_int * 4)(0, 300, 300, 1001), 4, 2, 128, 128) == 0      # empty prompt
+    assert lib.rbs_varlen_workspace_bytes(3, good, 4, 2, 64, 128) == 0                                          # head_dim
+    p = ctypes.c_void_p(0x1000)
+    t = _t()
+    assert lib.rbs_prefill_varlen(3, good, 4, 2, 128, 128, t, t, t, t, 0.22, 0.18, 1, 1, 1, p, p, need - 1, None) == WORKSPACE
+    assert lib.rbs_prefill_varlen(3, good, 4, 2, 128, 128, t, t, t, t, 0.22, 0.18, 1, 1, 1, None, p, need, None) == INVALID
+    assert lib.rbs_prefill_varlen(0, good, 4, 2, 128, 128, t, t, t, t, 0.22, 0.18, 1, 1, 1, p, p, need, None) == INVALID

@@ -415,6 +415,11 @@ def test_varlen_batch_equals_one_call_per_prompt():
         torch.cuda.synchronize()
         assert torch.equal(O[cu[k]:cu[k + 1]], O1[0])
         assert torch.equal(dens[k], d1)
+    # the same batch through the library's own varlen entry point (one call, one workspace)
+    from paper_2609_20971_b200.binding import rbs_prefill_varlen
+    O2, dens2 = rbs_prefill_varlen(Qp, Kp, Vp, cu, B)
+    torch.cuda.synchronize()
+    assert torch.equal(O2, O) and all(torch.equal(dens2[k:k + 1], dens[k]) for k in range(len(lens)))
     # oracle check on the shortest prompt (one short block: dense causal attention over 100 tokens)
     k = 2
     Q64, K64, V64 = (to_f64(t) for t in parts[k])
