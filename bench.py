@@ -30,7 +30,7 @@ import torch
 # DRAM bytes (read + write) of one rbs_sparse_prefill launch from an ncu capture of that workload at the default
 # thresholds: (bytes, where the capture is summarised).  A workload without a capture reports null and says so.
 NCU_TRAFFIC_BYTES = {
-    "q30b_128k": (4552352512 + 1036708096, "profiles/prefill_tc_kernel_traffic_q30b_128k.md"),
+    "q30b_128k": (4623220000 + 1038194000, "profiles/prefill_tc_kernel_q30b_128k.md"),
     "q30b_32k": (455600000 + 232200000, "profiles/prefill_tc_kernel_q30b_32k.md"),
 }
 NOMINAL_BF16_TFLOPS = 2250.0     # dense bf16 per B200, for context next to the measured peak
@@ -465,6 +465,25 @@ def run_ours(args):
             torch.cuda.synchronize()
             chunk[f"last_64_query_blocks_ms_{name}"] = e0.elapsed_time(e1) / 3
 
+    # group-shared masks (union over the G heads of a KV group): the one-head-per-CTA kernel on the union mask against
+    # the head-packed kernel (two heads per CTA over one K/V stream)
+    grouped = {}
+    if rank == 0 and B >= 128 and (cfg.Hq // cfg.Hkv) % 2 == 0 and args.detail == "full":
+        from paper_2609_20971_b200 import rbs_mask_group_union, rbs_sparse_prefill_grouped
+        mu, du = mask.clone(), density.clone()
+        rbs_mask_group_union(mu, du, cfg.Hkv, B, cfg.N)
+        for name, fn in (("one_head_per_cta", lambda: rbs_sparse_prefill(Qg, Kg, Vg, mu, B, out=Og)),
+                         ("two_heads_per_cta", lambda: rbs_sparse_prefill_grouped(Qg, Kg, Vg, mu, B, out=Og))):
+            fn()
+            torch.cuda.synchronize()
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            grouped[f"t_sparse_ms_{name}"] = e0.elapsed_time(e1)
+        grouped["density_of_union"] = float(du.float().mean().item())
+        del mu, du
+
     # threshold sweep of the headline config: the paper's three (alpha_base, alpha_rescue) pairs (Sec. 4.4 sensitivity
     # table) and pairs calibrated by bisection to realised densities of about 3 / 5 / 10 / 15 %, timed like the step
     sweep = []
@@ -575,6 +594,7 @@ def run_ours(args):
             "stats_us_times_sm_mhz": (t_stats_rot * 1e3 * stat_clocks["sm_mhz"]) if stat_clocks and stat_clocks.get("sm_mhz") else None,
             "peaks": peaks,
             "chunked_call": chunk,
+            "group_shared_masks": grouped,
             "sweep": sweep,
             "workloads": others,
             "bench_wall_s": time.time() - T_START,
