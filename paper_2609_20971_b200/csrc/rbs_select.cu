@@ -333,7 +333,10 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
 constexpr int kPairThreads = 576;
 constexpr int kPairProducer = 16, kPairMma = 17;
 
-template <int B>
+// HALVES (blocks of 256): the two "heads" of an item are the two halves of 128 tokens of ONE head's query block; the
+// sum over the block's tokens (Eq. block_aggregation) is then the sum of the two groups' sums, handed from the second
+// group to the first like the token halves inside a group; the first group alone keeps the scores and writes the mask.
+template <int B, bool HALVES>
 __global__ void __launch_bounds__(kPairThreads, 1)
 select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmChi,
                    const __grid_constant__ CUtensorMap tmClo, const SelectParams p, int n_items, int l_floats,
@@ -351,12 +354,15 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   __shared__ __align__(8) uint64_t bar_qfull[2], bar_qempty[2], bar_cfull[2], bar_cempty[2], bar_tfull[2][2], bar_tempty[2][2];
   __shared__ __align__(8) uint64_t bar_half[2][4][2];      // [head][lane quarter][tile parity]: second half's sums are there
   __shared__ __align__(8) float2 sHalf[2][4][2][32];       // the partial sums (base, rescue) of the second half
-  __shared__ float sRed[2][2][8], sRedQ[2][16];
+  __shared__ __align__(8) uint64_t bar_group[4][2];        // HALVES: the second group's sums are there
+  __shared__ __align__(8) float2 sGroup[4][2][32];
+  __shared__ float sRed[2][2][8], sRedQ[2][16], sQstat[2][2];
   __shared__ uint32_t s_tmem;
 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int Hkv = p.Hq / p.G, GP = p.G / 2;
+  const int Hkv = p.Hq / p.G, GP = HALVES ? p.G : p.G / 2;   // items per (batch, KV head, query block)
   const int per_i = p.L * Hkv * GP;
+  constexpr int QB = HALVES ? 2 * B : B;                     // tokens of a query block
 
   if (tid == 0) {
     for (int s = 0; s < 2; ++s) {
@@ -370,6 +376,7 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         mbar_init(smem_u32(&bar_tfull[hw][s]), 1); mbar_init(smem_u32(&bar_tempty[hw][s]), 8);
         for (int q = 0; q < 4; ++q) mbar_init(smem_u32(&bar_half[hw][q][s]), 1);
       }
+      for (int q = 0; q < 4; ++q) mbar_init(smem_u32(&bar_group[q][s]), 1);
     }
     mbar_fence_init();
   }
@@ -385,8 +392,11 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     int rem = w % per_i;
     const int pr = rem % GP; rem /= GP;
     hk = rem % Hkv; l = rem / Hkv;
-    h0 = hk * p.G + 2 * pr;
+    h0 = hk * p.G + (HALVES ? pr : 2 * pr);
   };
+  // tensor-memory columns of the accumulator of group hw, buffer buf (HALVES: the two groups' accumulators of a buffer
+  // side by side, so that they can be read as one row of 2 B tokens)
+  auto acc_col = [](int hw, uint32_t buf) -> uint32_t { return HALVES ? (buf * 2 + hw) * B : (hw * 2 + buf) * B; };
 
   if (warp == kPairProducer) {
     // ------------------------------- TMA producer -------------------------------
@@ -402,8 +412,9 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const uint32_t dst = smem_u32(sQ) + slot * 2 * kQTile, bar = smem_u32(&bar_qfull[slot]);
         mbar_arrive_expect_tx(bar, 2 * kQTile);
         for (int hw = 0; hw < 2; ++hw) {
-          tma_load_4d(dst + hw * kQTile, &tmQ, bar, 0, h0 + hw, il * B, l);
-          tma_load_4d(dst + hw * kQTile + kPanelQ, &tmQ, bar, 64, h0 + hw, il * B, l);
+          const int hq = HALVES ? h0 : h0 + hw, tok0 = HALVES ? il * QB + hw * B : il * B;
+          tma_load_4d(dst + hw * kQTile, &tmQ, bar, 0, hq, tok0, l);
+          tma_load_4d(dst + hw * kQTile + kPanelQ, &tmQ, bar, 64, hq, tok0, l);
         }
         ++nq;
       };
@@ -450,7 +461,7 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t d0 = tmem_base + buf * B, d1 = tmem_base + (2 + buf) * B;
+        const uint32_t d0 = tmem_base + acc_col(0, buf), d1 = tmem_base + acc_col(1, buf);
         mma_ss_k128_commit_elect(d0, dchi, dq0, kIdesc, kPanelC, kPanelQ, 0, 0);
         mma_ss_k128_commit_elect(d1, dchi, dq1, kIdesc, kPanelC, kPanelQ, smem_u32(&bar_cempty[0]), 0);
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_cfull[1]), nt & 1, status, kWaitTmaFull));
@@ -478,16 +489,26 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     for (int w = blockIdx.x; ok && w < n_items; w += gridDim.x, ++k) {
       int il, l, hk, h0;
       decode(w, il, l, hk, h0);
-      const int i = p.q0 + il, h = h0 + hw;
+      const int i = p.q0 + il, h = HALVES ? h0 : h0 + hw;
       const int n_tiles = i / 128 + 1;
       const int crow0 = static_cast<int>((static_cast<int64_t>(l) * Hkv + hk) * p.Mpad);
       const uint32_t slot = k & 1;
       const unsigned char* q = sQ + slot * 2 * kQTile + hw * kQTile;
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_qfull[slot]), (k >> 1) & 1, status, kWaitTmaFull));
-      const int n_tok = min(B, p.Nq - il * B);
+      const int n_tok = HALVES ? max(0, min(B, p.Nq - il * QB - hw * B)) : min(B, p.Nq - il * B);   // of this group
       float qn_max, qn_spread;
       ok = query_norm_shifts<B, 256>(q, wtid, n_tok, sQn_h, &sRedQ[hw][0], gbar, ok, qn_max, qn_spread);
       if (wtid == 0) mbar_arrive(smem_u32(&bar_qempty[slot]));      // the Q tile itself is not read again by this group
+      if (HALVES) {
+        // the norms' maximum and spread are those of the whole block of 2 B tokens: exchange with the other group
+        if (wtid == 0) { sQstat[hw][0] = qn_max; sQstat[hw][1] = n_tok > 0 ? qn_max - qn_spread : INFINITY; }
+        ok = group_all<512>(ok, 3);                                  // both groups (and a failed wait ends both)
+        const float g_max = fmaxf(sQstat[0][0], sQstat[1][0]), g_min = fminf(sQstat[0][1], sQstat[1][1]);
+        if (wtid < B) sQn_h[wtid] -= g_max - qn_max;                // shifts relative to the block's maximum
+        qn_max = g_max;
+        qn_spread = g_max - g_min;
+        ok = group_all<512>(ok, 3);                                  // shifts written; sQstat may be rewritten by the next item
+      }
       float mxb = -INFINITY, mxr = -INFINITY;     // running maxima of this thread's L values (causal blocks only)
       for (int bt = 0; ok && bt < n_tiles; ++bt, ++nt) {
         const uint32_t buf = nt & 1;
@@ -496,7 +517,7 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         tc_fence_after_sync();
         const int prow = crow0 + bt * 128 + row;
         const float gs = p.gs[prow], cn = p.cnorm[prow];
-        const uint32_t taddr = tmem_base + (hw * 2 + buf) * B + (static_cast<uint32_t>(wq * 32) << 16);
+        const uint32_t taddr = tmem_base + acc_col(hw, buf) + (static_cast<uint32_t>(wq * 32) << 16);
         // the decisions of score_tile, identical in the two warps that share these rows
         const float mb = qn_max * cn * 1.0001f;
         const bool no_rescue = __all_sync(0xffffffffu, gs == 0.f);
@@ -507,6 +528,7 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           __syncwarp();
           if (lane == 0) mbar_arrive(smem_u32(&bar_tempty[hw][buf]));
         };
+        const uint32_t gbar2 = smem_u32(&bar_group[wq][buf]);
         if (half == 1) {
           if (cheap) {
             float sb, sr;
@@ -515,20 +537,43 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           }
           release();                                  // (also orders the shared-memory writes before the arrival below)
           if (lane == 0) mbar_arrive(hbar);
+        } else if (HALVES && hw == 1) {
+          // second group, first token half: its group's sums go on to the first group
+          float sb = 0.f, sr = 0.f;
+          if (cheap) partial_sums<B, B / 2>(taddr, sQn_h, gs, -mb, no_rescue, n_tok, 0, sb, sr);
+          ok = __all_sync(0xffffffffu, mbar_wait(hbar, (nt >> 1) & 1, status, kWaitPReady));
+          if (cheap) {
+            const float2 o = sHalf[hw][wq][buf][lane];
+            sGroup[wq][buf][lane] = make_float2(sb + o.x, sr + o.y);
+          }
+          release();
+          if (lane == 0) mbar_arrive(gbar2);
         } else {
           float Lb, Lr;
           if (cheap) {
             float sb, sr;
             partial_sums<B, B / 2>(taddr, sQn_h, gs, -mb, no_rescue, n_tok, 0, sb, sr);
             ok = __all_sync(0xffffffffu, mbar_wait(hbar, (nt >> 1) & 1, status, kWaitPReady));
-            const float2 o = sHalf[hw][wq][buf][lane];
-            // the buffer (and with it this slot of sHalf) goes back only after the partner's sums have been taken
+            float2 o = sHalf[hw][wq][buf][lane];
+            if (HALVES) {
+              ok = __all_sync(0xffffffffu, ok && mbar_wait(gbar2, (nt >> 1) & 1, status, kWaitPReady));
+              const float2 o2 = sGroup[wq][buf][lane];
+              o.x += o2.x; o.y += o2.y;
+            }
+            // the buffer (and with it these slots of sHalf / sGroup) goes back only after the partners' sums have been taken
             release();
             Lb = mb + fast_log2(sb + o.x);
             Lr = no_rescue ? Lb : fmaf(qn_max, gs, mb) + fast_log2(sr + o.y);
           } else {
-            score_tile<B, false>(taddr, sQn_h, gs, cn, qn_max, qn_spread, n_tok, []() {}, Lb, Lr);
+            // exact shifts: this warp takes the whole row alone (HALVES: both groups' accumulators, side by side)
+            if (HALVES) {
+              const int n_all = min(QB, p.Nq - il * QB);
+              score_tile<QB, false>(taddr, sQn, gs, cn, qn_max, qn_spread, n_all, []() {}, Lb, Lr);
+            } else {
+              score_tile<B, false>(taddr, sQn_h, gs, cn, qn_max, qn_spread, n_tok, []() {}, Lb, Lr);
+            }
             ok = __all_sync(0xffffffffu, mbar_wait(hbar, (nt >> 1) & 1, status, kWaitPReady));
+            if (HALVES) ok = __all_sync(0xffffffffu, ok && mbar_wait(gbar2, (nt >> 1) & 1, status, kWaitPReady));
             release();
           }
           const int b = p.perm[prow];                 // the block this accumulator row belongs to
@@ -554,7 +599,7 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const int64_t mrow = ((static_cast<int64_t>(l) * p.Hq + h) * p.Mq + il) * p.W;
       const bool all_forced = i >= p.M - p.n_recent;
       unsigned int cnt = 0;
-      for (int wd = wg; ok && wd < p.W; wd += 8) {
+      for (int wd = wg; ok && !(HALVES && hw == 1) && wd < p.W; wd += 8) {
         const int b = wd * 32 + lane;
         const bool valid = b <= i;
         bool kb = false, kr = false, kf = false;
@@ -620,26 +665,29 @@ static rbs_status launch_select_tc(const SelectParams& p, const rbs_tensor& Q, c
 // (blocks of 256: two Q tiles of 64 KB each do not fit twice; an odd group size; very long rows).
 template <int B>
 static size_t pair_kernel_smem(const SelectParams& p, int* l_floats) {
-  if (B > 128 || p.G % 2 != 0) return 0;
+  if (B <= 128 && p.G % 2 != 0) return 0;
+  constexpr int BT = B > 128 ? 128 : B;     // tokens per Q tile (blocks of 256: two tiles of 128 of one head)
   *l_floats = (p.M + 127) / 128 * 128;
-  const size_t bytes = static_cast<size_t>(4) * 128 * 128 + 4 * 2 * static_cast<size_t>(B) * 128 + 2 * B * sizeof(float) +
+  const size_t bytes = static_cast<size_t>(4) * 128 * 128 + 4 * 2 * static_cast<size_t>(BT) * 128 + 2 * BT * sizeof(float) +
                        4 * static_cast<size_t>(*l_floats) * sizeof(float);
-  return bytes <= 227 * 1024 - 6 * 1024 ? bytes : 0;   // about 5 KB of static shared memory beside it
+  return bytes <= 227 * 1024 - 8 * 1024 ? bytes : 0;   // up to 7 KB of static shared memory beside it
 }
 
 template <int B>
 static rbs_status launch_select_pair(const SelectParams& p, const rbs_tensor& Q, size_t smem, int l_floats, cudaStream_t s) {
   CUtensorMap tmQ, tmChi, tmClo;
-  rbs_status st = make_tmap_lthd(&tmQ, Q.ptr, p.L, p.Nq, p.Hq, kHeadDim, Q.stride_batch, Q.stride_token, Q.stride_head, 64, B, true);
+  constexpr bool kHalves = B > 128;
+  constexpr int BT = kHalves ? 128 : B;
+  rbs_status st = make_tmap_lthd(&tmQ, Q.ptr, p.L, p.Nq, p.Hq, kHeadDim, Q.stride_batch, Q.stride_token, Q.stride_head, 64, BT, true);
   if (st != RBS_OK) return st;
   const int64_t rows = static_cast<int64_t>(p.L) * (p.Hq / p.G) * p.Mpad;
   if ((st = make_tmap_2d(&tmChi, p.chi, rows, kHeadDim, 64, 128)) != RBS_OK) return st;
   if ((st = make_tmap_2d(&tmClo, p.clo, rows, kHeadDim, 64, 128)) != RBS_OK) return st;
   unsigned int* status = device_status_ptr();
   if (status == nullptr) return RBS_ERR_CUDA;
-  auto kern = select_pair_kernel<B>;
+  auto kern = select_pair_kernel<BT, kHalves>;
   if ((st = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem)) != RBS_OK) return st;
-  const long long n_items = static_cast<long long>(p.L) * (p.Hq / 2) * p.Mq;
+  const long long n_items = static_cast<long long>(p.L) * (kHalves ? p.Hq : p.Hq / 2) * p.Mq;
   if (n_items > 0x7fffffffLL) return RBS_ERR_UNSUPPORTED;
   const int grid = static_cast<int>(n_items < sm_count() ? n_items : sm_count());
   kern<<<grid, kPairThreads, smem, s>>>(tmQ, tmChi, tmClo, p, static_cast<int>(n_items), l_floats, status);
@@ -709,7 +757,7 @@ static rbs_status select_impl(const rbs_shape* shape, int q_start_block, int n_q
   p.scale_log2 = scale_log2; p.t_base = log2f(alpha_base); p.t_rescue = log2f(alpha_rescue);
   p.n_sink = n_sink; p.n_local = n_local; p.n_recent = n_recent;
   p.mask = mask; p.dbg_base = dbg_base_mask; p.dbg_rescue = dbg_rescue_mask; p.counts = counts;
-  if (x.B == 256) st = launch_select_tc<256>(p, Q, s);
+  if (x.B == 256) st = launch_select<256>(p, Q, s);
   else st = (x.B == 128) ? launch_select<128>(p, Q, s) : launch_select<64>(p, Q, s);
   if (st != RBS_OK) return st;
   const int nh = x.L * x.Hq;

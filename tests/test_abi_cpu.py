@@ -166,3 +166,24 @@ def test_varlen_argument_checks(lib):
     assert lib.rbs_prefill_varlen(3, good, 4, 2, 128, 128, t, t, t, t, 0.22, 0.18, 1, 1, 1, p, p, need - 1, None) == WORKSPACE
     assert lib.rbs_prefill_varlen(3, good, 4, 2, 128, 128, t, t, t, t, 0.22, 0.18, 1, 1, 1, None, p, need, None) == INVALID
     assert lib.rbs_prefill_varlen(0, good, 4, 2, 128, 128, t, t, t, t, 0.22, 0.18, 1, 1, 1, p, p, need, None) == INVALID
+
+
+def test_grouped_prefill_and_box_selector_argument_checks(lib):
+    p = ctypes.c_void_p(0x1000)
+    t = _t()
+    lib.rbs_sparse_prefill_grouped.restype = ctypes.c_int
+    good = RbsShape(1, 1024, 4, 2, 128, 128)
+    assert lib.rbs_sparse_prefill_grouped(ctypes.byref(good), t, t, t, None, t, None, ctypes.c_float(0.0), None) == INVALID   # needs a mask
+    odd = RbsShape(1, 1024, 3, 1, 128, 128)                       # group of three heads: no pairs
+    assert lib.rbs_sparse_prefill_grouped(ctypes.byref(odd), t, t, t, p, t, None, ctypes.c_float(0.0), None) == UNSUPPORTED
+    b64 = RbsShape(1, 1024, 4, 2, 128, 64)
+    assert lib.rbs_sparse_prefill_grouped(ctypes.byref(b64), t, t, t, p, t, None, ctypes.c_float(0.0), None) == UNSUPPORTED
+    box = binding.RbsBox(0x1000, 0x1000)
+    need = lib.rbs_workspace_bytes(3, ctypes.byref(good))
+    assert need > 0 and lib.rbs_workspace_bytes(3, ctypes.byref(RbsShape(1, 1024, 4, 2, 128, 256))) == 0
+    call = lambda shape, delta, ws_bytes=need: lib.rbs_select_box(ctypes.byref(shape), t, box, ctypes.c_double(delta), 1, 1, 1, p, p,
+                                                                  None, p, ws_bytes, None)
+    assert call(good, 0.0) == INVALID and call(good, 1.5) == INVALID
+    assert call(good, 0.05, need - 1) == WORKSPACE
+    assert call(RbsShape(1, 1024, 4, 2, 128, 256), 0.05) == UNSUPPORTED
+    assert lib.rbs_block_stats_box(ctypes.byref(good), t, _stats(), binding.RbsBox(0, 0x1000), None) == INVALID
