@@ -24,10 +24,11 @@ __device__ __forceinline__ bool group_all(bool ok, int id) {
 // Query norms of one Q tile (B tokens, 128-byte-swizzled panels of 64 columns in shared memory), by the NT threads
 // of an epilogue group: sD[t] = ||q_t|| - max_t ||q_t|| (<= 0), and the maximum and the spread (max - min) of the norms
 // over the block's n_tok real tokens.  `red` is 2 * NT / 32 floats of scratch.  Two group barriers.
-template <int B, int NT>
+// PANEL_STRIDE: bytes from the first panel of the tile to the second.
+template <int B, int NT, uint32_t PANEL_STRIDE = B * 128>
 __device__ __forceinline__ bool query_norm_shifts(const unsigned char* q, int wtid, int n_tok, float* sD, float* red,
                                                   int bar_id, bool ok, float& qn_max, float& qn_spread) {
-  constexpr uint32_t kPanelQ = B * 128;
+  constexpr uint32_t kPanelQ = PANEL_STRIDE;
   constexpr int TPT = (B + NT - 1) / NT;   // tokens per thread
   constexpr int NWG = NT / 32;
   const int lane = wtid & 31, wq = wtid >> 5;
@@ -38,7 +39,7 @@ __device__ __forceinline__ bool query_norm_shifts(const unsigned char* q, int wt
     const int tok = wtid + u * NT;
     nrm[u] = 0.f;
     if (ok && tok < B) {
-      float s2 = 0.f;
+      float s2[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};   // eight independent chains of 32 terms
 #pragma unroll
       for (int c = 0; c < 16; ++c) {
         const uint4 v = *reinterpret_cast<const uint4*>(q + (c >> 3) * kPanelQ + tok * 128 + (((c & 7) ^ (tok & 7)) << 4));
@@ -46,11 +47,11 @@ __device__ __forceinline__ bool query_norm_shifts(const unsigned char* q, int wt
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const float a = bf16lo(wv[e]), c2 = bf16hi(wv[e]);
-          s2 = fmaf(a, a, s2);
-          s2 = fmaf(c2, c2, s2);
+          s2[2 * e] = fmaf(a, a, s2[2 * e]);
+          s2[2 * e + 1] = fmaf(c2, c2, s2[2 * e + 1]);
         }
       }
-      nrm[u] = sqrtf(s2);
+      nrm[u] = sqrtf(((s2[0] + s2[1]) + (s2[2] + s2[3])) + ((s2[4] + s2[5]) + (s2[6] + s2[7])));
       if (tok < n_tok) { mx = fmaxf(mx, nrm[u]); mn = fminf(mn, nrm[u]); }
     }
   }
@@ -195,24 +196,22 @@ __device__ __forceinline__ void score_tile(uint32_t taddr, const float* __restri
 
 
 // The single-pass case of score_tile for the columns [c_begin, c_begin + NC) of the accumulator row only:
-// sum_t 2^(x_t + c) and sum_t 2^(x_t + c + gs (||q_t|| - ||q||max)) over those tokens.
+// sum_t 2^(x_t + c) and sum_t 2^(x_t + c + gs (||q_t|| - ||q||max)) over those tokens.  The load of each chunk of 16
+// columns is in flight while the chunk before it is reduced.
 template <int B, int NC>
 __device__ __forceinline__ void partial_sums(uint32_t taddr, const float* __restrict__ sD, float gs, float c, bool no_rescue,
                                              int n_tok, int c_begin, float& sum_b, float& sum_r) {
+  static_assert(NC % 32 == 0, "chunks are taken in pairs");
   const uint64_t g2 = f2_pack(gs, gs), c2 = f2_pack(c, c);
   uint64_t sb_a = 0ull, sb_b = 0ull, sr_a = 0ull, sr_b = 0ull;
-#pragma unroll 1
-  for (int c0 = c_begin; c0 < c_begin + NC; c0 += 32) {
-    uint32_t r[32];
-    tmem_ld32(taddr + c0, r);
-    tmem_wait_ld();
+  auto chunk = [&](uint32_t (&r)[16], int c0) {
     if (n_tok < B) {
 #pragma unroll
-      for (int qq = 0; qq < 32; ++qq)
+      for (int qq = 0; qq < 16; ++qq)
         if (c0 + qq >= n_tok) r[qq] = 0xff800000u;   // -inf: tokens past the sequence end do not count
     }
 #pragma unroll
-    for (int j = 0; j < 32; j += 4) {
+    for (int j = 0; j < 16; j += 4) {
       const uint64_t e01 = f2_add(f2_pack(__uint_as_float(r[j]), __uint_as_float(r[j + 1])), c2);
       const uint64_t e23 = f2_add(f2_pack(__uint_as_float(r[j + 2]), __uint_as_float(r[j + 3])), c2);
       float e0, e1, e2, e3;
@@ -229,6 +228,17 @@ __device__ __forceinline__ void partial_sums(uint32_t taddr, const float* __rest
         sr_b = f2_add(sr_b, f2_pack(fast_exp2(f2), fast_exp2(f3)));
       }
     }
+  };
+  uint32_t ra[16], rb[16];
+  tmem_ld16(taddr + c_begin, ra);
+#pragma unroll 1
+  for (int c0 = c_begin; c0 < c_begin + NC; c0 += 32) {
+    tmem_wait_ld();
+    tmem_ld16(taddr + c0 + 16, rb);
+    chunk(ra, c0);
+    tmem_wait_ld();
+    if (c0 + 32 < c_begin + NC) tmem_ld16(taddr + c0 + 32, ra);
+    chunk(rb, c0 + 16);
   }
   float a0, a1, a2, a3;
   f2_unpack(f2_add(sb_a, sb_b), a0, a1);

@@ -345,13 +345,15 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   constexpr uint32_t kStage = 4 * kPanelC;         // hi panels 0,1 then lo panels 0,1
   constexpr uint32_t kPanelQ = B * 128;
   constexpr uint32_t kQTile = 2 * kPanelQ;         // one head's Q tile
-  constexpr uint32_t kIdesc = idesc_bf16_f32(128, B, false);
+  // the two heads' tiles are ONE operand of 2 B rows: a product with N = 2 B reads the centroid panel from shared
+  // memory once for both heads
+  constexpr uint32_t kIdesc = idesc_bf16_f32(128, 2 * B, false);
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* sC = smem;                                        // 64 KB
-  unsigned char* sQ = sC + kStage;                                 // [slot 2][head 2][kQTile]
+  unsigned char* sQ = sC + kStage;                                 // [slot 2][panel 2][head 2][kPanelQ]
   float* sQn = reinterpret_cast<float*>(sQ + 4 * kQTile);          // [head 2][B]
   float* sL = sQn + 2 * B;                                         // [head 2][branch 2][l_floats]
-  __shared__ __align__(8) uint64_t bar_qfull[2], bar_qempty[2], bar_cfull[2], bar_cempty[2], bar_tfull[2][2], bar_tempty[2][2];
+  __shared__ __align__(8) uint64_t bar_qfull[2], bar_qempty[2], bar_cfull[4], bar_cempty[4], bar_tfull[2][2], bar_tempty[2][2];
   __shared__ __align__(8) uint64_t bar_half[2][4][2];      // [head][lane quarter][tile parity]: second half's sums are there
   __shared__ __align__(8) float2 sHalf[2][4][2][32];       // the partial sums (base, rescue) of the second half
   __shared__ __align__(8) uint64_t bar_group[4][2];        // HALVES: the second group's sums are there
@@ -371,7 +373,8 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       // epilogue groups even reach it: without their arrivals the slot would be refilled under them, and the full
       // barrier could run two phases ahead of a waiter, which a parity wait cannot tell from no progress)
       mbar_init(smem_u32(&bar_qfull[s]), 1); mbar_init(smem_u32(&bar_qempty[s]), 3);
-      mbar_init(smem_u32(&bar_cfull[s]), 1); mbar_init(smem_u32(&bar_cempty[s]), 1);
+      mbar_init(smem_u32(&bar_cfull[s]), 1); mbar_init(smem_u32(&bar_cempty[s]), 1);        // one pair per 64-column
+      mbar_init(smem_u32(&bar_cfull[2 + s]), 1); mbar_init(smem_u32(&bar_cempty[2 + s]), 1);   // panel: hi 0, hi 1, lo 0, lo 1
       for (int hw = 0; hw < 2; ++hw) {
         mbar_init(smem_u32(&bar_tfull[hw][s]), 1); mbar_init(smem_u32(&bar_tempty[hw][s]), 8);
         for (int q = 0; q < 4; ++q) mbar_init(smem_u32(&bar_half[hw][q][s]), 1);
@@ -394,9 +397,9 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     hk = rem % Hkv; l = rem / Hkv;
     h0 = hk * p.G + (HALVES ? pr : 2 * pr);
   };
-  // tensor-memory columns of the accumulator of group hw, buffer buf (HALVES: the two groups' accumulators of a buffer
-  // side by side, so that they can be read as one row of 2 B tokens)
-  auto acc_col = [](int hw, uint32_t buf) -> uint32_t { return HALVES ? (buf * 2 + hw) * B : (hw * 2 + buf) * B; };
+  // tensor-memory columns of the accumulator of group hw, buffer buf: the two groups' accumulators of a buffer side by
+  // side (one product writes both; HALVES reads them as one row of 2 B tokens)
+  auto acc_col = [](int hw, uint32_t buf) -> uint32_t { return (buf * 2 + hw) * B; };
 
   if (warp == kPairProducer) {
     // ------------------------------- TMA producer -------------------------------
@@ -413,8 +416,8 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         mbar_arrive_expect_tx(bar, 2 * kQTile);
         for (int hw = 0; hw < 2; ++hw) {
           const int hq = HALVES ? h0 : h0 + hw, tok0 = HALVES ? il * QB + hw * B : il * B;
-          tma_load_4d(dst + hw * kQTile, &tmQ, bar, 0, hq, tok0, l);
-          tma_load_4d(dst + hw * kQTile + kPanelQ, &tmQ, bar, 64, hq, tok0, l);
+          tma_load_4d(dst + hw * kPanelQ, &tmQ, bar, 0, hq, tok0, l);
+          tma_load_4d(dst + hw * kPanelQ + kQTile, &tmQ, bar, 64, hq, tok0, l);
         }
         ++nq;
       };
@@ -427,14 +430,15 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const int crow0 = static_cast<int>((static_cast<int64_t>(l) * Hkv + hk) * p.Mpad);
         const uint32_t dst = smem_u32(sC);
         for (int bt = 0; ok && bt < n_tiles; ++bt, ++nc) {
-          if (nc > 0 && !mbar_wait(smem_u32(&bar_cempty[0]), (nc - 1) & 1, status, kWaitStageFree)) { ok = false; break; }
-          mbar_arrive_expect_tx(smem_u32(&bar_cfull[0]), kStage / 2);
-          tma_load_2d(dst, &tmChi, smem_u32(&bar_cfull[0]), 0, crow0 + bt * 128);
-          tma_load_2d(dst + kPanelC, &tmChi, smem_u32(&bar_cfull[0]), 64, crow0 + bt * 128);
-          if (nc > 0 && !mbar_wait(smem_u32(&bar_cempty[1]), (nc - 1) & 1, status, kWaitStageFree)) { ok = false; break; }
-          mbar_arrive_expect_tx(smem_u32(&bar_cfull[1]), kStage / 2);
-          tma_load_2d(dst + 2 * kPanelC, &tmClo, smem_u32(&bar_cfull[1]), 0, crow0 + bt * 128);
-          tma_load_2d(dst + 3 * kPanelC, &tmClo, smem_u32(&bar_cfull[1]), 64, crow0 + bt * 128);
+          // The four 64-column panels of a centroid tile (hi 0, hi 1, lo 0, lo 1) are separate pipeline slots: a panel
+          // of the NEXT tile is requested as soon as the products with that panel of this one are done, a quarter, a
+          // half, ... of the tile's tensor work before its end.
+          for (int q = 0; q < 4; ++q) {
+            if (nc > 0 && !mbar_wait(smem_u32(&bar_cempty[q]), (nc - 1) & 1, status, kWaitStageFree)) { ok = false; break; }
+            mbar_arrive_expect_tx(smem_u32(&bar_cfull[q]), kPanelC);
+            tma_load_2d(dst + q * kPanelC, q < 2 ? &tmChi : &tmClo, smem_u32(&bar_cfull[q]), (q & 1) * 64, crow0 + bt * 128);
+          }
+          if (!ok) break;
           // the next item's Q tiles go out right behind this item's first centroid tile
           if (bt == 0 && w + static_cast<int>(gridDim.x) < n_items) load_q(w + gridDim.x);
         }
@@ -443,7 +447,6 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
   } else if (warp == kPairMma) {
     // ------------------------------- MMA issuer -------------------------------
     const uint64_t dchi = smem_desc_sw128(smem_u32(sC), 16, 1024);
-    const uint64_t dclo = smem_desc_sw128(smem_u32(sC) + 2 * kPanelC, 16, 1024);
     uint32_t nt = 0, k = 0;      // centroid tiles and items processed so far
     bool ok = true;
     for (int w = blockIdx.x; ok && w < n_items; w += gridDim.x, ++k) {
@@ -451,8 +454,7 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const int n_tiles = (p.q0 + il) / 128 + 1;
       const uint32_t slot = k & 1;
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_qfull[slot]), (k >> 1) & 1, status, kWaitTmaFull));
-      const uint64_t dq0 = smem_desc_sw128(smem_u32(sQ) + slot * 2 * kQTile, 16, 1024);
-      const uint64_t dq1 = smem_desc_sw128(smem_u32(sQ) + slot * 2 * kQTile + kQTile, 16, 1024);
+      const uint64_t dq = smem_desc_sw128(smem_u32(sQ) + slot * 2 * kQTile, 16, 1024);
       for (int bt = 0; ok && bt < n_tiles; ++bt, ++nt) {
         const uint32_t buf = nt & 1;
         ok = mbar_wait(smem_u32(&bar_cfull[0]), nt & 1, status, kWaitTmaFull);
@@ -461,14 +463,19 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t d0 = tmem_base + acc_col(0, buf), d1 = tmem_base + acc_col(1, buf);
-        mma_ss_k128_commit_elect(d0, dchi, dq0, kIdesc, kPanelC, kPanelQ, 0, 0);
-        mma_ss_k128_commit_elect(d1, dchi, dq1, kIdesc, kPanelC, kPanelQ, smem_u32(&bar_cempty[0]), 0);
-        ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_cfull[1]), nt & 1, status, kWaitTmaFull));
+        const uint32_t d = tmem_base + acc_col(0, buf);
+        constexpr uint64_t kPanelQ16 = kQTile >> 4, kPanelC16 = kPanelC >> 4;   // panel strides in descriptor units
+        // panel q of the centroid tile times panel q & 1 of the two heads' Q tiles
+        for (int q = 0; q < 4; ++q) {
+          if (q > 0) {
+            ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_cfull[q]), nt & 1, status, kWaitTmaFull));
+            if (!ok) break;
+            tc_fence_after_sync();
+          }
+          mma_ss_k64_commit_elect(d, dchi + q * kPanelC16, dq + (q & 1) * kPanelQ16, kIdesc, smem_u32(&bar_cempty[q]), q > 0);
+        }
         if (!ok) break;
-        tc_fence_after_sync();
-        mma_ss_k128_commit_elect(d0, dclo, dq0, kIdesc, kPanelC, kPanelQ, smem_u32(&bar_tfull[0][buf]), 1);
-        mma_ss_k128_commit_elect(d1, dclo, dq1, kIdesc, kPanelC, kPanelQ, smem_u32(&bar_cempty[1]), 1);
+        mma_commit_elect(smem_u32(&bar_tfull[0][buf]));
         mma_commit_elect(smem_u32(&bar_tfull[1][buf]));
         if (bt == n_tiles - 1) mma_commit_elect(smem_u32(&bar_qempty[slot]));   // this item's Q tiles are free
       }
@@ -493,11 +500,11 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       const int n_tiles = i / 128 + 1;
       const int crow0 = static_cast<int>((static_cast<int64_t>(l) * Hkv + hk) * p.Mpad);
       const uint32_t slot = k & 1;
-      const unsigned char* q = sQ + slot * 2 * kQTile + hw * kQTile;
+      const unsigned char* q = sQ + slot * 2 * kQTile + hw * kPanelQ;
       ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_qfull[slot]), (k >> 1) & 1, status, kWaitTmaFull));
       const int n_tok = HALVES ? max(0, min(B, p.Nq - il * QB - hw * B)) : min(B, p.Nq - il * B);   // of this group
       float qn_max, qn_spread;
-      ok = query_norm_shifts<B, 256>(q, wtid, n_tok, sQn_h, &sRedQ[hw][0], gbar, ok, qn_max, qn_spread);
+      ok = query_norm_shifts<B, 256, kQTile>(q, wtid, n_tok, sQn_h, &sRedQ[hw][0], gbar, ok, qn_max, qn_spread);
       if (wtid == 0) mbar_arrive(smem_u32(&bar_qempty[slot]));      // the Q tile itself is not read again by this group
       if (HALVES) {
         // the norms' maximum and spread are those of the whole block of 2 B tokens: exchange with the other group
@@ -512,11 +519,13 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
       float mxb = -INFINITY, mxr = -INFINITY;     // running maxima of this thread's L values (causal blocks only)
       for (int bt = 0; ok && bt < n_tiles; ++bt, ++nt) {
         const uint32_t buf = nt & 1;
+        // the row's constants are requested before the wait for the accumulator: their latency passes under it
+        const int prow = crow0 + bt * 128 + row;
+        const float gs = __ldg(p.gs + prow), cn = __ldg(p.cnorm + prow);
+        const int b_row = __ldg(p.perm + prow);       // the block this accumulator row belongs to
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_tfull[hw][buf]), (nt >> 1) & 1, status, kWaitMmaDone));
         if (!ok) break;
         tc_fence_after_sync();
-        const int prow = crow0 + bt * 128 + row;
-        const float gs = p.gs[prow], cn = p.cnorm[prow];
         const uint32_t taddr = tmem_base + acc_col(hw, buf) + (static_cast<uint32_t>(wq * 32) << 16);
         // the decisions of score_tile, identical in the two warps that share these rows
         const float mb = qn_max * cn * 1.0001f;
@@ -576,7 +585,7 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             if (HALVES) ok = __all_sync(0xffffffffu, ok && mbar_wait(gbar2, (nt >> 1) & 1, status, kWaitPReady));
             release();
           }
-          const int b = p.perm[prow];                 // the block this accumulator row belongs to
+          const int b = b_row;
           if (b > i) { Lb = -INFINITY; Lr = -INFINITY; }
           sLb[b] = Lb;
           sLr[b] = Lr;
