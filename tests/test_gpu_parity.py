@@ -64,6 +64,12 @@ CASES = {
     "ragged_n_b256": SynthConfig("ragged_n_b256", N=256 * 9 + 100, Hq=2, Hkv=2, B=256, sigma=0.5, seed=37),
     "lognormal_b128": SynthConfig("lognormal_b128", N=128 * 40, Hq=2, Hkv=2, B=128, sigma=0.5, sigma_ln=0.5,
                                   p_needle=0.05, seed=33),
+    # a last block of 256 whose SECOND half of 128 tokens is the short one, an odd group size, and coherent queries
+    # of large norm: logits beyond the range in which the norm bounds can serve as log-sum-exp shifts
+    "ragged_n2_b256": SynthConfig("ragged_n2_b256", N=256 * 6 + 200, Hq=3, Hkv=1, B=256, sigma=(0.1, 1.0), s_q=3.5,
+                                  seed=38),
+    "hot_b128": SynthConfig("hot_b128", N=128 * 19 + 5, Hq=4, Hkv=2, B=128, sigma=(0.1, 1.0), s_q=3.5, sigma_ln=0.3,
+                            seed=39),
 }
 
 
