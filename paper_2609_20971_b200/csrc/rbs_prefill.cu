@@ -282,9 +282,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
     mbar_fence_init();
     // the Q tile does not depend on the mask: it is on its way before tensor memory is set up and the mask row is read
     // (4.06 / 6.29 / 9.62 against 4.13 / 6.34 / 9.68 ms at 3 / 5 / 8 % density)
+    // Q is read exactly once per launch: evict-first, so that it does not push the K/V of the KV head in flight out
+    // of L2 (-0.2 % of the launch)
     mbar_arrive_expect_tx(smem_u32(&bar_q), kTile);
-    tma_load_4d(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, Tl * B, l);
-    tma_load_4d(smem_u32(sQ + kPanel), &tmQ, smem_u32(&bar_q), 64, h, Tl * B, l);
+    const uint64_t pol_q = make_policy_evict_first();
+    tma_load_4d_hint(smem_u32(sQ), &tmQ, smem_u32(&bar_q), 0, h, Tl * B, l, pol_q);
+    tma_load_4d_hint(smem_u32(sQ + kPanel), &tmQ, smem_u32(&bar_q), 64, h, Tl * B, l, pol_q);
   }
   if (warp == 5) tmem_alloc(smem_u32(&s_tmem), 256);
   tc_fence_before_sync();
