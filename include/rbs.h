@@ -45,7 +45,8 @@ typedef enum {
   RBS_ERR_UNSUPPORTED = 2, /* shape outside the supported set listed above */
   RBS_ERR_WORKSPACE = 3,   /* workspace missing or smaller than rbs_workspace_bytes() */
   RBS_ERR_CUDA = 4,        /* a CUDA runtime / driver call failed (launch, tensor-map encode, ...) */
-  RBS_ERR_TIMEOUT = 5      /* a bounded device-side wait gave up  */
+  RBS_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up  */
+  RBS_ERR_DEBUG_CHECK = 6  /* debug build only: a device-side index check failed (rbs_device_status) */
 } rbs_status;
 
 typedef struct {
@@ -291,7 +292,10 @@ RBS_API rbs_status rbs_prefill_varlen(int n_prompts, const int* cu_seqlens, int 
  * iteration limit.  A wait that runs out records a non-zero code in a device-side status word, lets the
  * kernel drain and return, and leaves the CUDA context usable; outputs of that launch are then
  * undefined.  This call synchronises `stream`, reads the word into *code_out (nullable) and, if
- * `clear` is non-zero, resets it.  Returns RBS_OK when the word is 0, RBS_ERR_TIMEOUT otherwise.
+ * `clear` is non-zero, resets it.  Returns RBS_OK when the word is 0, RBS_ERR_TIMEOUT for a wait that ran out
+ * (codes 1 .. 7: which kind of wait) and RBS_ERR_DEBUG_CHECK for a failed index check of the debug build
+ * (code 0x100 + site; the library built with -DRBS_DEBUG checks the indices of its writes and of its
+ * tile walks and skips an access that fails; the release build has no such checks).
  * (No counterpart in the paper: an operational check.)
  */
 RBS_API rbs_status rbs_device_status(void* stream, unsigned int* code_out, int clear);

@@ -29,6 +29,15 @@ RBS_API int rbs_selftest_device_table(void);
  */
 RBS_API rbs_status rbs_selftest_wait_timeout(unsigned int spin_limit, unsigned int* gave_up, void* stream);
 
+/*
+ * Debug build only (the library compiled with -DRBS_DEBUG; rbs_version() says "debug checks"): launches one thread
+ * on `stream` that runs one of the kernels' index checks with an index equal to its bound.  The check fails, records
+ * 0x100 + 0xff in the device status word and the guarded access is skipped: afterwards *skipped (device, one
+ * uint32) is 1, rbs_device_status() reports RBS_ERR_DEBUG_CHECK until cleared, and the CUDA context is fully usable
+ * (nothing traps or faults).  The release build has no such checks and returns RBS_ERR_UNSUPPORTED without a launch.
+ */
+RBS_API rbs_status rbs_selftest_debug_check(unsigned int* skipped, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -13,7 +13,9 @@ from dataclasses import dataclass
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "librbs_b200.so")
+# RBS_DEBUG=1 in the environment selects the library built with -DRBS_DEBUG (device-side index checks that are
+# reported through rbs_device_status; `python -m paper_2609_20971_b200.build --debug`)
+LIB_PATH = os.path.join(_PKG, "librbs_b200_debug.so" if os.environ.get("RBS_DEBUG", "0") not in ("", "0") else "librbs_b200.so")
 
 RBS_OP_BLOCK_STATS, RBS_OP_SELECT, RBS_OP_SPARSE_PREFILL, RBS_OP_SELECT_BOX = 0, 1, 2, 3
 SELECTOR_RBS, SELECTOR_CENTROID_ONLY, SELECTOR_FULL_L2 = 0, 1, 2
@@ -92,6 +94,8 @@ def load_library() -> ctypes.CDLL:
     lib.rbs_selftest_device_table.argtypes = []
     lib.rbs_selftest_wait_timeout.restype = i
     lib.rbs_selftest_wait_timeout.argtypes = [ctypes.c_uint, vp, vp]
+    lib.rbs_selftest_debug_check.restype = i
+    lib.rbs_selftest_debug_check.argtypes = [vp, vp]
     lib.rbs_status_string.restype = ctypes.c_char_p
     lib.rbs_status_string.argtypes = [i]
     lib.rbs_version.restype = ctypes.c_char_p
@@ -155,7 +159,7 @@ def rbs_device_status(clear: bool = True) -> int:
     kernel gave up (the outputs of that launch are then undefined).  `clear` resets the word."""
     code = ctypes.c_uint(0)
     rc = load_library().rbs_device_status(_stream(), ctypes.byref(code), 1 if clear else 0)
-    if rc not in (0, 5):
+    if rc not in (0, 5, 6):     # a recorded time-out or failed debug check is the answer, not a failure of the call
         _check(rc, "rbs_device_status")
     return int(code.value)
 
@@ -166,6 +170,22 @@ def rbs_selftest_wait_timeout(spin_limit: int = 4096) -> torch.Tensor:
     flag = torch.zeros(1, dtype=torch.int32, device="cuda")
     _check(load_library().rbs_selftest_wait_timeout(spin_limit, _ptr(flag), _stream()), "rbs_selftest_wait_timeout")
     return flag
+
+
+def rbs_selftest_debug_check() -> torch.Tensor | None:
+    """Debug library only (RBS_DEBUG=1): runs one device-side index check that fails by construction and returns
+    the device flag the guarded access leaves (1 = skipped); the status word then holds 0x1ff.  None in the
+    release library, which has no such checks."""
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    rc = load_library().rbs_selftest_debug_check(_ptr(flag), _stream())
+    if rc == 2:       # RBS_ERR_UNSUPPORTED: release build
+        return None
+    _check(rc, "rbs_selftest_debug_check")
+    return flag
+
+
+def rbs_version() -> str:
+    return load_library().rbs_version().decode()
 
 
 def rbs_block_stats(K: torch.Tensor, block: int, stats: BlockStats | None = None) -> BlockStats:

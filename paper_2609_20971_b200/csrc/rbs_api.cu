@@ -83,8 +83,15 @@ extern "C" const char* rbs_status_string(rbs_status status) {
     case RBS_ERR_WORKSPACE: return "RBS_ERR_WORKSPACE";
     case RBS_ERR_CUDA: return "RBS_ERR_CUDA";
     case RBS_ERR_TIMEOUT: return "RBS_ERR_TIMEOUT";
+    case RBS_ERR_DEBUG_CHECK: return "RBS_ERR_DEBUG_CHECK";
   }
   return "RBS_ERR_UNKNOWN";
 }
 
-extern "C" const char* rbs_version(void) { return "rbs-b200 0.1 (sm_100a)"; }
+extern "C" const char* rbs_version(void) {
+#ifdef RBS_DEBUG
+  return "rbs-b200 0.1 (sm_100a, debug checks)";
+#else
+  return "rbs-b200 0.1 (sm_100a)";
+#endif
+}

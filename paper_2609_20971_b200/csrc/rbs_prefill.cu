@@ -266,6 +266,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
   const int i = T / R;                      // its query block
   const int h = hk * p.G + rem % p.G;
   if (Tl * 128 >= p.Nq) return;             // a tile wholly past the end of the queries (short last block of 256)
+  if (!RBS_DBG_OK(i >= p.q0 && i - p.q0 < p.Mq && h < p.Hq && l < p.L && T < p.M * R, status, kDbgPrefillTile)) return;
   const uint32_t* mrow = p.mask ? p.mask + ((static_cast<int64_t>(l) * p.Hq + h) * p.Mq + (i - p.q0)) * p.W : nullptr;
   const int Tw = SCHED ? min(T, item.z - 1) : T;   // last sub-block this CTA may attend (T itself for a whole row)
   const int kb0 = SCHED ? item.y - 1 : -1;         // where the walk over the mask row starts
@@ -305,6 +306,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
       int b = next_kb(mrow, kb0, i, R, Tw);
       if (b < 0) mbar_wait(smem_u32(&bar_q), 0, status, kWaitTmaFull);   // nothing selected: the Q tile still has to land before the CTA may go
       for (int j = 0; b >= 0; ++j, b = next_kb(mrow, b, i, R, Tw)) {
+        if (!RBS_DBG_OK(b <= Tw && b * B < p.N, status, kDbgPrefillBlock)) break;
         if (j > 0 && !mbar_wait(smem_u32(&bar_s), (j - 1) & 1, status, kWaitStageFree)) break;   // S_{j-1} done: K free
         mbar_arrive_expect_tx(smem_u32(&bar_kfull), kTile);
         tma_load_4d(smem_u32(sK), &tmK, smem_u32(&bar_kfull), 0, hk, b * B, l);
@@ -544,7 +546,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant
         tma_store_commit();
         tma_store_wait_read();
       }
-      if (lse_dst && in_seq && o_ready) *lse_dst = (m_used + fast_log2(l_sum)) * 0.6931471805599453f;
+      if (lse_dst && in_seq && o_ready && RBS_DBG_OK(Tl * B + row < p.Nq, status, kDbgPrefillLse)) *lse_dst = (m_used + fast_log2(l_sum)) * 0.6931471805599453f;
     }
   }
   tc_fence_before_sync();

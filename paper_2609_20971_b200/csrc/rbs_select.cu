@@ -268,8 +268,10 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
         if (lane == 0) mbar_arrive(smem_u32(&bar_tempty[buf]));
       }, Lb, Lr);
       const bool causal = b <= i;
-      sLb[b] = causal ? Lb : -INFINITY;
-      sLr[b] = causal ? Lr : -INFINITY;
+      if (RBS_DBG_OK(b >= 0 && b < p.Mpad, status, kDbgSelectPerm)) {
+        sLb[b] = causal ? Lb : -INFINITY;
+        sLr[b] = causal ? Lr : -INFINITY;
+      }
     }
   }
   tc_fence_before_sync();
@@ -305,7 +307,7 @@ select_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant_
     }
     const uint32_t wb = __ballot_sync(0xffffffffu, kb), wr = __ballot_sync(0xffffffffu, kr);
     const uint32_t wf = __ballot_sync(0xffffffffu, kf);
-    if (lane == 0) {
+    if (lane == 0 && RBS_DBG_OK(mrow >= 0 && mrow + w < static_cast<int64_t>(p.L) * p.Hq * p.Mq * p.W, status, kDbgSelectMask)) {
       const uint32_t word = wb | wr | wf;
       p.mask[mrow + w] = word;
       if (p.dbg_base) p.dbg_base[mrow + w] = wb;
@@ -521,11 +523,13 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         const uint32_t buf = nt & 1;
         // the row's constants are requested before the wait for the accumulator: their latency passes under it
         const int prow = crow0 + bt * 128 + row;
-        const float gs = __ldg(p.gs + prow), cn = __ldg(p.cnorm + prow);
-        const int b_row = __ldg(p.perm + prow);       // the block this accumulator row belongs to
+        const bool prow_ok = RBS_DBG_OK(prow >= 0 && prow < p.L * Hkv * p.Mpad, status, kDbgSelectCentroid);
+        const float gs = prow_ok ? __ldg(p.gs + prow) : 0.f, cn = prow_ok ? __ldg(p.cnorm + prow) : 0.f;
+        const int b_row = prow_ok ? __ldg(p.perm + prow) : 0x7fffffff;   // the block this accumulator row belongs to
         ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bar_tfull[hw][buf]), (nt >> 1) & 1, status, kWaitMmaDone));
         if (!ok) break;
         tc_fence_after_sync();
+        (void)RBS_DBG_OK(acc_col(hw, buf) + B <= 4u * B, status, kDbgSelectTmem);
         const uint32_t taddr = tmem_base + acc_col(hw, buf) + (static_cast<uint32_t>(wq * 32) << 16);
         // the decisions of score_tile, identical in the two warps that share these rows
         const float mb = qn_max * cn * 1.0001f;
@@ -587,8 +591,10 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
           }
           const int b = b_row;
           if (b > i) { Lb = -INFINITY; Lr = -INFINITY; }
-          sLb[b] = Lb;
-          sLr[b] = Lr;
+          if (RBS_DBG_OK(b >= 0 && b < l_floats && b < p.Mpad, status, kDbgSelectPerm)) {
+            sLb[b] = Lb;
+            sLr[b] = Lr;
+          }
           mxb = fmaxf(mxb, Lb);
           mxr = fmaxf(mxr, Lr);
         }
@@ -619,7 +625,7 @@ select_pair_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
         const uint32_t wb = __ballot_sync(0xffffffffu, kb), wr = __ballot_sync(0xffffffffu, kr);
         const uint32_t wf = __ballot_sync(0xffffffffu, kf);
-        if (lane == 0) {
+        if (lane == 0 && RBS_DBG_OK(mrow >= 0 && mrow + wd < static_cast<int64_t>(p.L) * p.Hq * p.Mq * p.W, status, kDbgSelectMask)) {
           const uint32_t word = wb | wr | wf;
           p.mask[mrow + wd] = word;
           if (p.dbg_base) p.dbg_base[mrow + wd] = wb;

@@ -57,6 +57,32 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, unsigne
   return mbar_wait_limit(bar, parity, status, code, kSpinLimit);
 }
 
+// Debug build (-DRBS_DEBUG): index checks in the kernels.  A failing check records 0x100 + its site in the device
+// status word (first failure wins), the caller skips the access and the kernel runs on: no trap, the context stays
+// usable and rbs_device_status reports RBS_ERR_DEBUG_CHECK with the site.  In the release build the macro is the
+// constant `true` and its condition is not even compiled.
+enum DebugSite : unsigned int {
+  kDbgStatsRow = 1,        // block statistics: output row past the end of centroid / radius
+  kDbgSelectScore = 2,     // selector: score slot past the end of the row's L arrays in shared memory
+  kDbgSelectPerm = 3,      // selector: block index of an accumulator row outside the padded row count
+  kDbgSelectMask = 4,      // selector: mask word past the end of the mask
+  kDbgSelectTmem = 5,      // selector: accumulator columns past the allocated tensor memory
+  kDbgSelectCentroid = 6,  // selector: centroid row of a tile past the padded centroid arrays
+  kDbgPrefillBlock = 7,    // attention: key sub-block after the query tile or past the sequence
+  kDbgPrefillTile = 8,     // attention: query tile outside this call's queries
+  kDbgPrefillPart = 9,     // attention: partial-result slot outside the workspace
+  kDbgPrefillLse = 10,     // attention: lse index past the end
+};
+#ifdef RBS_DEBUG
+__device__ __forceinline__ bool dbg_record(bool cond, unsigned int* status, unsigned int site) {
+  if (!cond) atomicCAS(status, 0u, 0x100u + site);
+  return cond;
+}
+#define RBS_DBG_OK(cond, status, site) ::rbs::dbg_record((cond), (status), (site))
+#else
+#define RBS_DBG_OK(cond, status, site) true
+#endif
+
 // ------------------------------------------------------------------------------------------- TMA
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(map)) : "memory");

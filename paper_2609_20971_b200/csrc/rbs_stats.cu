@@ -122,8 +122,9 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
     }
     const float4 cen = make_float4(a0 * inv_rows, a1 * inv_rows, a2 * inv_rows, a3 * inv_rows);
     const int64_t blk = (static_cast<int64_t>(l) * Hkv + hk) * M + b;
-    if (part == 0) reinterpret_cast<float4*>(centroid + blk * kHeadDim)[lane] = cen;
-    if (BOX && part == 0) {
+    const bool row_ok = RBS_DBG_OK(blk < n_tiles && b * B < N, status, kDbgStatsRow);
+    if (part == 0 && row_ok) reinterpret_cast<float4*>(centroid + blk * kHeadDim)[lane] = cen;
+    if (BOX && part == 0 && row_ok) {
       reinterpret_cast<float4*>(box_lo + blk * kHeadDim)[lane] = make_float4(lo0, lo1, lo2, lo3);
       reinterpret_cast<float4*>(box_hi + blk * kHeadDim)[lane] = make_float4(hi0, hi1, hi2, hi3);
     }
@@ -175,10 +176,10 @@ block_stats_warp_kernel(const __grid_constant__ CUtensorMap tmK, int n_tiles, in
       if (lane == 0) s_max[warp] = rmax;
       mbar_arrive(smem_u32(&pair_bar[group]));
       pair_ok = mbar_wait(smem_u32(&pair_bar[group]), 1, status, kWaitStageFree) && pair_ok;
-      if (part == 0 && lane == 0) radius[blk] = sqrtf(fmaxf(rmax, s_max[warp ^ 1]));
+      if (part == 0 && lane == 0 && row_ok) radius[blk] = sqrtf(fmaxf(rmax, s_max[warp ^ 1]));
       if (!__all_sync(0xffffffffu, pair_ok)) break;
     } else {
-      if (lane == 0) radius[blk] = sqrtf(rmax);
+      if (lane == 0 && row_ok) radius[blk] = sqrtf(rmax);
     }
   }
 }

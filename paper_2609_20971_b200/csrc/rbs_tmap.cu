@@ -103,6 +103,15 @@ rbs_status ensure_dynamic_smem(const void* kernel, size_t bytes) {
 }
 
 // One CTA, one thread: waits on an mbarrier that nothing ever arrives on, with the given probe limit.
+#ifdef RBS_DEBUG
+// one thread runs a debug check that fails by construction (the "index" 1 against a bound of 1)
+__global__ void selftest_debug_check_kernel(unsigned int* status, unsigned int* skipped) {
+  const int index = 1, bound = 1;
+  if (RBS_DBG_OK(index < bound, status, 0xffu)) *skipped = 0u;   // the guarded "access"
+  else *skipped = 1u;
+}
+#endif
+
 __global__ void selftest_wait_kernel(unsigned int* status, unsigned int spin_limit, unsigned int* gave_up) {
   __shared__ __align__(8) uint64_t bar;
   mbar_init(smem_u32(&bar), 1);
@@ -123,7 +132,7 @@ extern "C" rbs_status rbs_device_status(void* stream, unsigned int* code_out, in
     if (cudaMemcpyToSymbol(rbs::g_device_status, &zero, sizeof(zero)) != cudaSuccess) return RBS_ERR_CUDA;
   }
   if (code_out) *code_out = code;
-  return code == 0 ? RBS_OK : RBS_ERR_TIMEOUT;
+  return code == 0 ? RBS_OK : (code >= 0x100u ? RBS_ERR_DEBUG_CHECK : RBS_ERR_TIMEOUT);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -160,4 +169,17 @@ extern "C" rbs_status rbs_selftest_wait_timeout(unsigned int spin_limit, unsigne
   rbs::selftest_wait_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(status, spin_limit, gave_up);
   RBS_CUDA_OK(cudaGetLastError());
   return RBS_OK;
+}
+
+extern "C" rbs_status rbs_selftest_debug_check(unsigned int* skipped, void* stream) {
+#ifdef RBS_DEBUG
+  if (skipped == nullptr) return RBS_ERR_INVALID_ARG;
+  unsigned int* status = rbs::device_status_ptr();
+  if (status == nullptr) return RBS_ERR_CUDA;
+  rbs::selftest_debug_check_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(status, skipped);
+  return cudaGetLastError() == cudaSuccess ? RBS_OK : RBS_ERR_CUDA;
+#else
+  (void)skipped; (void)stream;
+  return RBS_ERR_UNSUPPORTED;   // the release build has no device-side checks
+#endif
 }

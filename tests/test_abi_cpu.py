@@ -40,7 +40,24 @@ def test_every_declared_symbol_is_exported(lib):
 def test_status_strings_and_version(lib):
     assert lib.rbs_status_string(0) == b"RBS_OK"
     assert lib.rbs_status_string(2) == b"RBS_ERR_UNSUPPORTED"
-    assert b"sm_100a" in lib.rbs_version()
+    assert lib.rbs_status_string(6) == b"RBS_ERR_DEBUG_CHECK"
+    assert b"sm_100a" in lib.rbs_version() and b"debug" not in lib.rbs_version()
+
+
+def test_debug_library_builds_and_exports_the_same_symbols():
+    """The variant with device-side index checks (-DRBS_DEBUG) is the same ABI: every declared symbol, and a version
+    string that says which variant is loaded.  (Its checks run in the GPU tests.)"""
+    import ctypes
+    from paper_2609_20971_b200.build import build_library
+    dbg = ctypes.CDLL(build_library(debug=True))
+    for n in declared_functions():
+        assert hasattr(dbg, n), n
+    dbg.rbs_version.restype = ctypes.c_char_p
+    assert b"debug checks" in dbg.rbs_version()
+    # the self-test refuses a null flag before any launch (no GPU needed)
+    dbg.rbs_selftest_debug_check.restype = ctypes.c_int
+    dbg.rbs_selftest_debug_check.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+    assert dbg.rbs_selftest_debug_check(None, None) == INVALID
 
 
 def _t(ptr=0x1000, sb=0, st=128, sh=128):

@@ -1,0 +1,80 @@
+"""The library built with -DRBS_DEBUG (device-side index checks, reported through rbs_device_status) against the
+release library: the whole path runs clean under the checks and gives bit-identical results, and a check that fails is
+recorded and its access skipped without a trap or a fault.
+
+The debug library is selected by RBS_DEBUG=1 when the binding is imported, so it runs in a child process.
+"""
+import os
+import subprocess
+import sys
+
+import pytest
+import torch
+
+from paper_2609_20971_b200 import rbs_block_stats, rbs_select, rbs_sparse_prefill
+from paper_2609_20971_b200.binding import rbs_selftest_debug_check, rbs_version
+from paper_2609_20971_b200.synth import SynthConfig, make_inputs
+
+pytestmark = pytest.mark.gpu
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+CASES = [
+    dict(name="dbg_b64", N=64 * 70 + 9, Hq=2, Hkv=1, B=64, sigma=0.5, seed=91),
+    dict(name="dbg_b128", L=2, N=128 * 37 + 50, Hq=4, Hkv=2, B=128, sigma=(0.1, 1.0), seed=92),
+    dict(name="dbg_b256", N=256 * 7 + 200, Hq=3, Hkv=1, B=256, sigma=(0.1, 1.0), s_q=3.5, seed=93),
+]
+
+CHILD = r"""
+import sys, torch
+from paper_2609_20971_b200 import rbs_block_stats, rbs_select, rbs_sparse_prefill, rbs_device_status
+from paper_2609_20971_b200.binding import rbs_version, rbs_selftest_debug_check
+from paper_2609_20971_b200.synth import SynthConfig, make_inputs
+assert "debug checks" in rbs_version(), rbs_version()
+cases = eval(sys.argv[1]); out = {}
+for kw in cases:
+    cfg = SynthConfig(**kw)
+    Q, K, V = (t.cuda() for t in make_inputs(cfg))
+    st = rbs_block_stats(K, cfg.B)
+    mask, dens = rbs_select(Q, st, cfg.B, cfg.alpha_base, cfg.alpha_rescue, 1, 1, 1)
+    O = rbs_sparse_prefill(Q, K, V, mask, cfg.B)
+    Od = rbs_sparse_prefill(Q, K, V, None, cfg.B)
+    assert rbs_device_status(clear=True) == 0, "a device-side check or wait failed on " + cfg.name
+    out[cfg.name] = dict(centroid=st.centroid.cpu(), radius=st.radius.cpu(), mask=mask.cpu(), O=O.cpu(), Od=Od.cpu())
+# a check that fails by construction: recorded, its access skipped, nothing traps, and the library works afterwards
+flag = rbs_selftest_debug_check()
+code = rbs_device_status(clear=True)
+assert flag is not None and int(flag.item()) == 1 and code == 0x1ff, (flag, hex(code))
+cfg = SynthConfig(**cases[0])
+Q, K, V = (t.cuda() for t in make_inputs(cfg))
+st = rbs_block_stats(K, cfg.B)
+assert rbs_device_status(clear=True) == 0
+assert torch.equal(st.centroid.cpu(), out[cfg.name]["centroid"])
+torch.save(out, sys.argv[2])
+print("debug child ok")
+"""
+
+
+def test_release_library_has_no_device_checks():
+    assert "debug" not in rbs_version()
+    assert rbs_selftest_debug_check() is None
+
+
+def test_debug_library_runs_the_path_clean_and_bit_identical(tmp_path):
+    dump = str(tmp_path / "debug_out.pt")
+    env = dict(os.environ, RBS_DEBUG="1", PYTHONPATH=ROOT + os.pathsep + os.environ.get("PYTHONPATH", ""))
+    r = subprocess.run([sys.executable, "-c", CHILD, repr(CASES), dump], env=env, cwd=ROOT, capture_output=True,
+                       text=True, timeout=600)
+    assert r.returncode == 0 and "debug child ok" in r.stdout, r.stdout[-2000:] + r.stderr[-4000:]
+    got = torch.load(dump)
+    for kw in CASES:
+        cfg = SynthConfig(**kw)
+        Q, K, V = (t.cuda() for t in make_inputs(cfg))
+        st = rbs_block_stats(K, cfg.B)
+        mask, _ = rbs_select(Q, st, cfg.B, cfg.alpha_base, cfg.alpha_rescue, 1, 1, 1)
+        O = rbs_sparse_prefill(Q, K, V, mask, cfg.B)
+        Od = rbs_sparse_prefill(Q, K, V, None, cfg.B)
+        g = got[cfg.name]
+        assert torch.equal(st.centroid.cpu(), g["centroid"]) and torch.equal(st.radius.cpu(), g["radius"])
+        assert torch.equal(mask.cpu(), g["mask"])
+        assert torch.equal(O.cpu(), g["O"]) and torch.equal(Od.cpu(), g["Od"])
