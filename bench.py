@@ -587,7 +587,7 @@ def run_ours(args):
             "dense_tflops": dense_useful / (t_dense * 1e-3) / 1e12,
             "dense_tensor_frac": dense_useful / (t_dense * 1e-3) / 1e12 / peaks["tflops"],
             "stats_rotating_us": t_stats_rot * 1e3, "stats_rotating_us_launched_from_python": t_stats_rot_python * 1e3,
-            "stats_timing": "CUDA-graph replay of 4 launches over rotating K buffers, CUDA events around 2000 replays",
+            "stats_timing": "CUDA-graph replay of 4 launches over rotating K buffers, CUDA events bracketing 2000 replays",
             "stats_gbs": stats_gbs, "stats_hbm_frac": stats_gbs / peaks["hbm_gbs"],
             "stats_target": TARGET_HBM_FRAC, "stats_target_met": bool(stats_gbs / peaks["hbm_gbs"] >= TARGET_HBM_FRAC),
             "stats_clocks": stat_clocks,
