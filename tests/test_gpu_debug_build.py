@@ -61,6 +61,8 @@ def test_release_library_has_no_device_checks():
 
 
 def test_debug_library_runs_the_path_clean_and_bit_identical(tmp_path):
+    from paper_2609_20971_b200.build import build_library
+    build_library(debug=True)          # only compiles when the debug library is missing or older than its sources
     dump = str(tmp_path / "debug_out.pt")
     env = dict(os.environ, RBS_DEBUG="1", PYTHONPATH=ROOT + os.pathsep + os.environ.get("PYTHONPATH", ""))
     r = subprocess.run([sys.executable, "-c", CHILD, repr(CASES), dump], env=env, cwd=ROOT, capture_output=True,
